@@ -1,0 +1,409 @@
+#!/usr/bin/env python
+"""Benchmark of the DSGD-CECA hot path: fused SGD step + one CECA gossip round per iteration.
+
+Default workload ("resnet50_step"): n = 100 agents, d = 25,557,032 parameters per agent (a
+ResNet-50-sized flat vector), fp32, CECA-2P, X0 = Y0 ~ N(0, 0.01^2), G ~ N(0, 0.01^2), gamma = 0.1,
+updated in place.  A step is one call of ceca_gossip_sgd_step for iteration k (k keeps counting,
+so the steps cycle through all tau = 7 rounds of the CECA sequence).
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload NAME]
+
+Prints ONE JSON line (rank 0).  `value` is agent-parameter updates per second summed over all
+ranks, inputs resident in HBM; `e2e` is the same metric through ceca_gossip_sgd_step_host with
+pinned HOST buffers (copies inside the timed region); `roofline` is the dominant kernel's
+algorithmic bytes over its CUDA-event time against the measured copy bandwidth;
+`cpu_baseline` is the fp64 oracle timed on the host cores on a column slice.
+
+With N > 1 (torchrun) every rank runs the same workload on its own GPU: the update never mixes
+columns, so ranks are independent column blocks and there is no collective on the data path.
+"""
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "agent-param updates/s (n*d per gossip+SGD step)"
+UNIT = "agent-param updates/s"
+
+# name -> (kind, n, d, variant, extra)
+WORKLOADS = {
+    # the configuration the headline metric is quoted on
+    "resnet50_step": dict(kind="step", n=100, d=25_557_032, variant=2, gamma=0.1),
+    # smaller cases of the same kernels, for profiler captures and quick looks
+    "resnet18_step": dict(kind="step", n=24, d=11_689_512, variant=1, gamma=0.1),
+    "step_small": dict(kind="step", n=100, d=2_097_152, variant=2, gamma=0.1),
+    "consensus_fused": dict(kind="consensus", n=97, d=1 << 20, variant=2, fused=1),
+    "consensus_rounds": dict(kind="consensus", n=97, d=1 << 20, variant=2, fused=0),
+    "logreg_grad": dict(kind="logreg", n=63, m=2000, d=4096, variant=2, gamma=0.01),
+}
+
+FALLBACK_HBM_GBS = 6650.0
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
+# capture summarised under profiles/ (None until captured, or once the kernel has changed since).
+NCU_TRAFFIC_BYTES_PER_LAUNCH = {}
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.rows, self.proc, self.thread = [], None, None
+        self.cmd = ["nvidia-smi", "-i", str(index), "--query-gpu=" + self.FIELDS, "--format=csv,noheader,nounits",
+                    "-lms", "100"]
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(self.cmd, stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            return
+        self.thread = threading.Thread(target=self._read, daemon=True)
+        self.thread.start()
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def stop(self):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        self.thread.join(timeout=2)
+        sm = [float(r[0]) for r in self.rows if len(r) >= 6 and r[0].replace(".", "").isdigit()]
+        mx = [float(r[1]) for r in self.rows if len(r) >= 6 and r[1].replace(".", "").isdigit()]
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        reasons = [nm for j, nm in enumerate(names) if any(len(r) >= 6 and r[2 + j].lower() == "active" for r in self.rows)]
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": reasons, "samples": len(sm)}
+
+
+def dist_setup(n_gpus):
+    """(rank, world, local_rank, dist or None).  Under torchrun the ranks meet over NCCL (gloo without GPUs)."""
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if world == 1:
+        return 0, 1, 0, None
+    import torch
+    import torch.distributed as dist
+    os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+    backend = "nccl" if torch.cuda.is_available() else "gloo"
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if backend == "nccl":
+        torch.cuda.set_device(local_rank)
+    dist.init_process_group(backend=backend)
+    return dist.get_rank(), world, local_rank, dist
+
+
+def max_over_ranks(ms, dist, device):
+    """The slowest rank's time (device timing, max over ranks)."""
+    if dist is None:
+        return ms
+    import torch
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t[0])
+
+
+# ------------------------------------------------------------------------------------------------
+# the oracle on the host cores (cpu_baseline leg and --impl reference)
+# ------------------------------------------------------------------------------------------------
+
+def oracle_step_throughput(n, variant, gamma, cols, steps, threads=None):
+    import numpy as np
+    import oracle
+    import synthetic_inputs as synth
+    threads = threads or len(os.sched_getaffinity(0))
+    oracle.set_threads(threads)
+    x, y, g = synth.step_inputs(n, cols, seed=0, x_std=0.01, g_std=0.01)
+    x, y, g = x.numpy().astype(np.float64), y.numpy().astype(np.float64), g.numpy().astype(np.float64)
+    oracle.step(x, y, g, gamma, variant, 0)  # untimed: loads the library, touches the pages
+    t0 = time.perf_counter()
+    for k in range(steps):
+        x, y = oracle.step(x, y, g, gamma, variant, k)
+    dt = time.perf_counter() - t0
+    return n * cols * steps / dt, dt / steps, threads
+
+
+def run_reference(args, wl, rank, world):
+    """--impl reference: the fp64 oracle, as it stands, on the host cores, on a column slice."""
+    if rank != 0:
+        return
+    cols = min(wl["d"], 262_144)
+    per_step = []
+    for _ in range(args.warmup):
+        oracle_step_throughput(wl["n"], wl["variant"], wl["gamma"], cols, 1)
+    value, sec_per_step, threads = oracle_step_throughput(wl["n"], wl["variant"], wl["gamma"], cols, args.steps)
+    sample = "%d-column slice of the %d columns, all %d rows, %d steps; columns are independent, cost is linear in d" % (
+        cols, wl["d"], wl["n"], args.steps)
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": sec_per_step * 1e3, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": args.workload, "n_agents": wl["n"], "d": wl["d"], "variant": "2P" if wl["variant"] == 2 else "1P",
+                       "sample_columns": cols},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+# ------------------------------------------------------------------------------------------------
+# GPU legs
+# ------------------------------------------------------------------------------------------------
+
+def algorithmic_bytes_step(n, d, reads_y):
+    """x, e (and y unless its weight is zero) read once; x+, y+ written once; 4 bytes each."""
+    return (20 if reads_y else 16) * n * d
+
+
+def bench_step(args, wl, device, dist):
+    import torch
+    import paper_2306_00256_b200 as ceca
+    import synthetic_inputs as synth
+
+    n, d, variant, gamma = wl["n"], wl["d"], wl["variant"], wl["gamma"]
+    X, Y, G = synth.step_inputs(n, d, seed=0, x_std=0.01, g_std=0.01, device=device)
+    stream = torch.cuda.current_stream()
+    tau = ceca.ceca_schedule(n, variant, 0, peers=False)[0].tau
+    k = 0
+    for _ in range(args.warmup):
+        ceca.ceca_gossip_sgd_step(X, Y, G, gamma, variant, k)
+        k += 1
+    events = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
+    k_first = k
+    sampler = ClockSampler(torch.cuda.current_device())
+    sampler.start()
+    if dist is not None:
+        dist.barrier()
+    torch.cuda.synchronize()
+    events[0].record(stream)
+    for s in range(args.steps):
+        ceca.ceca_gossip_sgd_step(X, Y, G, gamma, variant, k)
+        k += 1
+        events[s + 1].record(stream)
+    torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+    clocks = sampler.stop()
+    total_ms = events[0].elapsed_time(events[-1])
+    per_launch = [events[s].elapsed_time(events[s + 1]) for s in range(args.steps)]
+    # dominant kernel: the launches that read Y (every round but r = 0), 20 B per agent-parameter
+    dominant = [per_launch[s] for s in range(args.steps)
+                if ceca.ceca_schedule(n, variant, k_first + s, peers=False)[0].b_num != 0
+                or ceca.ceca_schedule(n, variant, k_first + s, peers=False)[0].payload == 1]
+    launches = args.steps * (1 if d % 4 == 0 else 2)
+    roof = None
+    if dominant:
+        avg_ms = sum(dominant) / len(dominant)
+        peak, which = measured_peak()
+        achieved = algorithmic_bytes_step(n, d, True) / (avg_ms * 1e-3) / 1e9
+        roof = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH.get(args.workload),
+                "kernel": "step_walk_kernel<float4, gradient, reads Y>", "peak_source": "of " + which,
+                "avg_launch_ms": avg_ms, "launches_timed": len(dominant),
+                "frac_of_nominal_8TBs": achieved / 8000.0}
+    del X, Y, G
+    torch.cuda.empty_cache()
+    return total_ms, launches, roof, clocks, {"tau": tau, "in_place": True, "l2": "inputs (3 x n x d fp32) far larger than L2"}
+
+
+def bench_step_e2e(args, wl, device):
+    """The same iteration through ceca_gossip_sgd_step_host: pinned host X, Y, G; copies timed."""
+    import torch
+    import paper_2306_00256_b200 as ceca
+    import synthetic_inputs as synth
+    n, d, variant, gamma = wl["n"], wl["d"], wl["variant"], wl["gamma"]
+    try:
+        hx = torch.empty((n, d), dtype=torch.float32, pin_memory=True)
+        hy = torch.empty((n, d), dtype=torch.float32, pin_memory=True)
+        hg = torch.empty((n, d), dtype=torch.float32, pin_memory=True)
+        pinned = True
+    except RuntimeError:
+        hx, hy, hg = (torch.empty((n, d), dtype=torch.float32) for _ in range(3))
+        pinned = False
+    # fill the host buffers from the device generator, one row at a time
+    row = torch.empty(d, dtype=torch.float32, device=device)
+    gen = torch.Generator(device=device)
+    gen.manual_seed(0)
+    for i in range(n):
+        hx[i].copy_(row.normal_(std=0.01, generator=gen))
+    hy.copy_(hx)
+    for i in range(n):
+        hg[i].copy_(row.normal_(std=0.01, generator=gen))
+    del row
+    ws = torch.empty(3 << 30, dtype=torch.uint8, device=device)
+    steps = max(1, min(args.steps, args.e2e_steps))
+    k = 0
+    for _ in range(1):
+        ceca.ceca_gossip_sgd_step_host(hx, hy, hg, gamma, variant, k, ws)
+        k += 1
+    h2d = d2h = 0
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        rd = ceca.ceca_schedule(n, variant, k, peers=False)[0]
+        reads_y = rd.b_num != 0 or rd.payload == 1
+        ceca.ceca_gossip_sgd_step_host(hx, hy, hg, gamma, variant, k, ws)
+        h2d += (3 if reads_y else 2) * n * d * 4
+        d2h += 2 * n * d * 4
+        k += 1
+    torch.cuda.synchronize()
+    dt = time.perf_counter() - t0
+    return {"value": n * d * steps / dt, "unit": UNIT, "h2d_bytes_per_step": h2d // steps, "d2h_bytes_per_step": d2h // steps,
+            "steps": steps, "ms_per_step": dt / steps * 1e3, "pinned": pinned,
+            "api": "ceca_gossip_sgd_step_host (column slabs streamed through a 3 GiB device workspace)"}
+
+
+def bench_consensus(args, wl, device, dist):
+    import torch
+    import paper_2306_00256_b200 as ceca
+    import synthetic_inputs as synth
+    n, d, variant, fused = wl["n"], wl["d"], wl["variant"], wl["fused"]
+    X = synth.consensus_inputs(n, d, seed=1, device=device)
+    Xo, Yo = torch.empty_like(X), torch.empty_like(X)
+    ws = torch.zeros(64, dtype=torch.int32, device=device)
+    tau = ceca.ceca_schedule(n, variant, 0, peers=False)[0].tau
+    stream = torch.cuda.current_stream()
+    for _ in range(args.warmup):
+        ceca.ceca_consensus_rounds(X, None, variant, 0, tau, fused, X_out=Xo, Y_out=Yo, workspace=ws)
+    sampler = ClockSampler(torch.cuda.current_device())
+    sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    e0.record(stream)
+    for _ in range(args.steps):
+        ceca.ceca_consensus_rounds(X, None, variant, 0, tau, fused, X_out=Xo, Y_out=Yo, workspace=ws)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    total_ms = e0.elapsed_time(e1)
+    assert ceca.ceca_read_status(ws) == 0
+    peak, which = measured_peak()
+    per_elem = 12 if fused else (16 * tau - 4)   # fused: X in, X and Y out; per round: 16 B (12 B in round 0)
+    achieved = per_elem * n * d / (total_ms / args.steps * 1e-3) / 1e9
+    roof = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak, "traffic": None,
+            "kernel": "consensus_fused_kernel" if fused else "step_walk_kernel<float4, no gradient> x tau",
+            "peak_source": "of " + which}
+    launches = args.steps * (1 if fused else tau)
+    return total_ms, launches, roof, clocks, {"tau": tau, "rounds_per_step": tau,
+                                               "l2": "X is 407 MB, larger than L2; outputs go to separate buffers"}
+
+
+def bench_logreg(args, wl, device, dist):
+    import torch
+    import paper_2306_00256_b200 as ceca
+    import synthetic_inputs as synth
+    n, m, d, variant, gamma = wl["n"], wl["m"], wl["d"], wl["variant"], wl["gamma"]
+    A, L, _ = synth.logreg_problem(n, m, d, seed=3, flip=0.05, hetero_std=0.5, device=device)
+    X = torch.zeros(n, d, device=device); Y = torch.zeros(n, d, device=device); G = torch.empty(n, d, device=device)
+    ws = torch.empty(ceca.ceca_workspace_bytes(ceca.WS_LOGREG_GRAD, n, m, d), dtype=torch.uint8, device=device)
+    stream = torch.cuda.current_stream()
+    k = 0
+    for _ in range(args.warmup):
+        ceca.dsgd_logreg_grad(A, L, X, Y, k, variant, G, ws)
+        ceca.ceca_gossip_sgd_step(X, Y, G, gamma, variant, k)
+        k += 1
+    sampler = ClockSampler(torch.cuda.current_device())
+    sampler.start()
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(2 * args.steps + 1)]
+    torch.cuda.synchronize()
+    ev[0].record(stream)
+    for s in range(args.steps):
+        ceca.dsgd_logreg_grad(A, L, X, Y, k, variant, G, ws)
+        ev[2 * s + 1].record(stream)
+        ceca.ceca_gossip_sgd_step(X, Y, G, gamma, variant, k)
+        ev[2 * s + 2].record(stream)
+        k += 1
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    total_ms = ev[0].elapsed_time(ev[-1])
+    grad_ms = sum(ev[2 * s].elapsed_time(ev[2 * s + 1]) for s in range(args.steps)) / args.steps
+    peak, which = measured_peak()
+    achieved = (4 * n * m * d + 8 * n * d + 4 * n * m) / (grad_ms * 1e-3) / 1e9
+    roof = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak, "traffic": None,
+            "kernel": "logreg_fused_kernel + logreg_reduce_kernel", "peak_source": "of " + which, "avg_launch_ms": grad_ms}
+    return total_ms, 3 * args.steps, roof, clocks, {"m": m, "l2": "A is 2.06 GB, larger than L2"}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=70)
+    ap.add_argument("--warmup", type=int, default=7)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="resnet50_step", choices=sorted(WORKLOADS))
+    ap.add_argument("--e2e-steps", type=int, default=7)
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    wl = WORKLOADS[args.workload]
+
+    if args.impl == "reference":
+        rank = int(os.environ.get("RANK", "0"))
+        if wl["kind"] != "step":
+            if rank == 0:
+                print(json.dumps({"impl": "reference", "unavailable": "the reference arm times the step workloads only"}))
+            return
+        run_reference(args, wl, rank, int(os.environ.get("WORLD_SIZE", "1")))
+        return
+
+    import torch
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    rank, world, local_rank, dist = dist_setup(args.gpus)
+    torch.cuda.set_device(local_rank)
+    device = "cuda:%d" % local_rank
+    import paper_2306_00256_b200 as ceca
+    ceca.library()
+
+    fn = {"step": bench_step, "consensus": bench_consensus, "logreg": bench_logreg}[wl["kind"]]
+    total_ms, launches, roof, clocks, extra = fn(args, wl, device, dist)
+    total_ms = max_over_ranks(total_ms, dist, device)
+    units_per_step = wl["n"] * wl["d"]
+    value = world * units_per_step * args.steps / (total_ms * 1e-3)
+
+    e2e = None
+    if wl["kind"] == "step" and not args.no_e2e:
+        e2e = bench_step_e2e(args, wl, device)
+        if dist is not None:
+            ms = max_over_ranks(e2e["ms_per_step"], dist, device)
+            e2e["ms_per_step"] = ms
+            e2e["value"] = world * units_per_step / (ms * 1e-3)
+
+    cpu = None
+    if rank == 0 and world == 1 and wl["kind"] == "step" and not args.no_cpu_baseline:
+        cols = min(wl["d"], 262_144)
+        v, sec, threads = oracle_step_throughput(wl["n"], wl["variant"], wl["gamma"], cols, 3 * extra["tau"])
+        cpu = {"value": v, "unit": UNIT, "cores": threads, "kind": "oracle",
+               "sample": "%d-column slice (all %d rows), %d steps = 3 cycles of the CECA sequence, fp64" % (cols, wl["n"], 3 * extra["tau"])}
+
+    if rank == 0:
+        config = {"workload": args.workload, "n_agents": wl["n"], "d": wl["d"], "variant": "2P" if wl["variant"] == 2 else "1P"}
+        config.update(extra)
+        line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+                "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+                "dtype": "f32", "data": "synthetic", "config": config, "clocks": clocks, "gpu_launches": launches,
+                "e2e": e2e, "roofline": roof, "cpu_baseline": cpu}
+        print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,174 @@
+/*
+ * ceca.h -- C ABI of the DSGD-CECA hot path for one NVIDIA B200 (sm_100a).
+ *
+ * n simulated agents are the rows of dense row-major fp32 matrices X (the models x_i),
+ * Y (the auxiliary models y_i) and G (the stochastic gradients e_i), each n x d with a
+ * leading dimension ld >= d counted in elements.  One call applies one iteration of
+ * DSGD-CECA (Algorithm 1), or several CECA consensus rounds (Algorithm 2), to all agents.
+ *
+ * Conventions shared by every entry point
+ *   - Agent indices are 0-based: the paper's agent p is row p-1, so a "paper-odd" agent
+ *     is an even row.
+ *   - Pointers named X, Y, G, A, labels, *_out and workspace are DEVICE pointers unless the
+ *     function name ends in _host.  The caller owns every buffer; the library allocates no
+ *     device memory, keeps no global state between calls and never frees anything.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
+ *     Device entry points only enqueue work: they do not synchronise and return as soon
+ *     as the launches are queued.
+ *   - Argument errors are reported synchronously, before anything is launched, through the
+ *     return value.  Nothing aborts or traps; no exception crosses this boundary.
+ *   - `variant` is CECA_1P (pairwise exchange, even n only) or CECA_2P (send to one agent,
+ *     receive from another; any n >= 1).
+ *   - `k` is the iteration counter of Algorithm 1; the round is r = k mod tau with
+ *     tau = ceil(log2 n).  k may be any value in [0, 2^63).
+ */
+#ifndef CECA_H_
+#define CECA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum { CECA_1P = 1, CECA_2P = 2 } ceca_variant_t;
+
+typedef enum {
+  CECA_OK = 0,
+  CECA_ERR_INVALID_ARG = 1, /* NULL where data is needed, n < 1, d < 1, ld < d, k < 0, ...       */
+  CECA_ERR_ODD_N_1P = 2,    /* CECA-1P is defined for even n only (Sec. 3.2)                     */
+  CECA_ERR_ALIGNMENT = 3,   /* the fused consensus kernel needs 16-byte aligned rows             */
+  CECA_ERR_UNSUPPORTED = 4, /* e.g. in-place aliasing of only one of X/Y, fused path with n > 256 */
+  CECA_ERR_WORKSPACE = 5,   /* workspace NULL or smaller than ceca_workspace_bytes says          */
+  CECA_ERR_CUDA = 6         /* a CUDA runtime / driver call failed (launch, copy, map encode)    */
+} ceca_status_t;
+
+/*
+ * Everything Algorithm 1 derives from (n, k) for one iteration.
+ * Sec. 3.1 "Auxiliary variables": n-1 = (delta_0 ... delta_{tau-1})_2 with delta_0 the most
+ * significant digit; n_0 = 0, n_{r+1} = 2 n_r + delta_r.
+ * Algorithm 1: delta_r = 1 -> the message is built from x, a = 1/2, b = n_r/(2 n_r + 1);
+ *              delta_r = 0 -> the message is built from y, a = (n_r+1)/(2 n_r+1), b = 1/2.
+ * n = 1 (not covered by the paper): tau = 0, r = 0, a = b = 1, nobody to talk to.
+ */
+typedef struct {
+  int32_t n, tau, r, delta, n_r;
+  int32_t payload;                    /* 0: z = x (delta = 1);  1: z = y (delta = 0)          */
+  int32_t a_num, a_den, b_num, b_den; /* exact weights (not necessarily in lowest terms)      */
+  double a, b;                        /* a_num/a_den, b_num/b_den: one IEEE division each     */
+} ceca_round_t;
+
+/*
+ * Host function.  The CECA schedule of iteration k:
+ *   round      (out, may be NULL)  the scalars above;
+ *   recv_from  (out, host, int32[n], may be NULL)  agent i receives the message of recv_from[i];
+ *   send_to    (out, host, int32[n], may be NULL)  agent i sends its message to send_to[i].
+ * recv_from is the row-to-column map of the permutation matrix P^(k) = Q^(r):
+ *   CECA-2P, Eq. (2p-gossip-matrix-d1/d0): recv_from[i] = (i - n_r - delta_r) mod n;
+ *   CECA-1P, Eq. (1p-gossip-matrix): even row i <-> row (i + 2 n_r + 1) mod n.
+ * Errors: CECA_ERR_INVALID_ARG (n < 1, k < 0, bad variant), CECA_ERR_ODD_N_1P.
+ */
+ceca_status_t ceca_schedule(int32_t n, ceca_variant_t variant, int64_t k, ceca_round_t *round,
+                            int32_t *recv_from, int32_t *send_to);
+
+/*
+ * One DSGD-CECA iteration for all agents, Eq. (x-iter-dsgd) and Eq. (y-iter-dsgd):
+ *   u_i   = z_i - gamma e_i                         (the message of agent i; never stored)
+ *   x+_i  = a (x_i - gamma e_i) + (1 - a) u_{recv_from[i]}
+ *   y+_i  = b (y_i - gamma e_i) + (1 - b) u_{recv_from[i]}
+ * X, Y, G: device, n x d fp32, leading dimension ld.  G may be NULL (treated as zero: a pure
+ * CECA round of Sec. 3.1 / 3.2).  Y may be NULL only when the round ignores it (r = 0, where
+ * b = 0 and z = x).
+ * X_out, Y_out: device, same shape and ld.  Distinct buffers (ping-pong), or X_out == X and/or
+ * Y_out == Y (in place: every element is read and then written by the same thread).  A crossed
+ * alias (X_out == Y, Y_out == X, an output equal to G, X_out == Y_out) is CECA_ERR_UNSUPPORTED;
+ * partially overlapping buffers are not detected and give undefined results.
+ * fp32 arithmetic; a, b and 1-a, 1-b are formed in fp64 on the host and rounded once.
+ */
+ceca_status_t ceca_gossip_sgd_step(const float *X, const float *Y, const float *G, float *X_out,
+                                   float *Y_out, int32_t n, int64_t d, int64_t ld, float gamma,
+                                   ceca_variant_t variant, int64_t k, void *stream);
+
+/*
+ * `rounds` consecutive CECA rounds k0, k0+1, ..., k0+rounds-1 on (I, J) = (X, Y)
+ * (Sec. 3.1 "Main recursions", Algorithm 2; Sec. 3.2 for the 1-port pairing).
+ * After tau rounds that start at a multiple of tau every row of X_out is the column mean of
+ * X and row i of Y_out is the mean of the other n-1 rows (Appendix B.2, Lemma "matrix
+ * consensus"); one more round makes Y_out the mean as well.
+ *
+ *   fused = 0: one kernel launch per round, each a full pass over HBM.  Works for every n, d,
+ *              ld and alignment.  Y_out == NULL is allowed when workspace holds n*ld floats.
+ *   fused = 1: a single launch.  A column tile of all n rows is brought into shared memory by
+ *              TMA (cp.async.bulk.tensor), every round runs on chip, and the tile is written
+ *              back once.  Needs n <= 256, X / X_out (and Y / Y_out when used) 16-byte aligned
+ *              with ld*4 a multiple of 16 (else CECA_ERR_ALIGNMENT), ld < 2^32, rounds <= 64,
+ *              and a workspace of ceca_workspace_bytes(CECA_WS_CONSENSUS_FUSED, ...) bytes
+ *              whose first int32 is a status word: it is left unchanged when the launch
+ *              completes normally and set non-zero if a bounded on-chip wait for a TMA
+ *              transfer ran out (read it with ceca_read_status).  Y may be NULL when the
+ *              first round is r = 0; Y_out may be NULL.
+ * X_out == X (and Y_out == Y) in place is allowed in both modes.
+ */
+ceca_status_t ceca_consensus_rounds(const float *X, const float *Y, float *X_out, float *Y_out,
+                                    int32_t n, int64_t d, int64_t ld, ceca_variant_t variant,
+                                    int64_t k0, int32_t rounds, int32_t fused, void *workspace,
+                                    size_t workspace_bytes, void *stream);
+
+/*
+ * Per-agent logistic-regression gradient, the e^(k) of Algorithm 1 for the synthetic
+ * classification workloads (the paper leaves f_i generic, Eq. (opt-problem-setting); this
+ * particular loss is the benchmark's choice and has no counterpart in the paper):
+ *   f_i(w)   = (1/m) sum_s log(1 + exp(-l_s <a_s, w>)),  l_s in {-1, +1}
+ *   G[i, :]  = -(1/m) sum_s l_s sigma(-l_s <a_s, z_i>) a_s
+ * evaluated at the model Algorithm 1 selects in iteration k: z = X if delta_r = 1, else Y.
+ * A: device, n x m x d fp32, dense (sample rows contiguous, row stride d);
+ * labels: device, n x m fp32 holding -1 or +1;  X, Y, G: device, n x d with leading dimension ld.
+ * workspace: device, at least ceca_workspace_bytes(CECA_WS_LOGREG_GRAD, n, m, d) bytes; holds
+ * per-block partial sums that a second, fixed-order pass adds up, so results are identical from
+ * run to run.
+ */
+ceca_status_t dsgd_logreg_grad(const float *A, const float *labels, const float *X, const float *Y,
+                               int64_t k, float *G, int32_t n, int32_t m, int64_t d, int64_t ld,
+                               ceca_variant_t variant, void *workspace, size_t workspace_bytes,
+                               void *stream);
+
+typedef enum {
+  CECA_WS_CONSENSUS_FUSED = 1,    /* ceca_consensus_rounds, fused = 1                      */
+  CECA_WS_CONSENSUS_UNFUSED = 2,  /* ceca_consensus_rounds, fused = 0 with Y_out == NULL   */
+  CECA_WS_LOGREG_GRAD = 3,        /* dsgd_logreg_grad                                      */
+  CECA_WS_STEP_HOST = 4           /* ceca_gossip_sgd_step_host: the smallest useful size   */
+} ceca_workspace_kind_t;
+
+/* Host function.  Minimum workspace size in bytes for the call named by `kind`
+ * (m is ignored except for CECA_WS_LOGREG_GRAD; pass ld for d where rows are padded). */
+size_t ceca_workspace_bytes(ceca_workspace_kind_t kind, int32_t n, int32_t m, int64_t d);
+
+/*
+ * Host function.  Waits for `stream`, then copies the int32 status word at the start of a
+ * fused-consensus workspace into *status_out (0 = no bounded wait ran out).  Zero the word
+ * (cudaMemsetAsync) before the first launch that uses the workspace.
+ */
+ceca_status_t ceca_read_status(const void *workspace, int32_t *status_out, void *stream);
+
+/*
+ * The same iteration as ceca_gossip_sgd_step for callers whose data lives in HOST memory
+ * (pinned memory gives full copy bandwidth; pageable memory works but is slower).
+ * X, Y (updated in place) and G are host pointers, n x d with leading dimension ld.  Columns
+ * never interact in the update, so the call cuts the columns into slabs, and for each slab
+ * copies X, Y, G to the device, runs the step kernel in place and copies X, Y back, with the
+ * copies and the kernels of neighbouring slabs overlapping on internal streams.
+ * workspace: DEVICE memory, workspace_bytes >= ceca_workspace_bytes(CECA_WS_STEP_HOST, n, 0, d);
+ * more workspace means wider slabs.  The call returns after all slabs have been written back.
+ */
+ceca_status_t ceca_gossip_sgd_step_host(float *X, float *Y, const float *G, int32_t n, int64_t d,
+                                        int64_t ld, float gamma, ceca_variant_t variant, int64_t k,
+                                        void *workspace, size_t workspace_bytes);
+
+/* Host function.  A short English name for a status code (static storage). */
+const char *ceca_status_string(ceca_status_t status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CECA_H_ */

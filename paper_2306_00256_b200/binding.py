@@ -1,0 +1,194 @@
+"""ctypes binding of include/ceca.h.  Argument marshalling only."""
+import ctypes
+import os
+
+import numpy as np
+
+from . import build as _build
+
+CECA_1P = 1
+CECA_2P = 2
+WS_CONSENSUS_FUSED = 1
+WS_CONSENSUS_UNFUSED = 2
+WS_LOGREG_GRAD = 3
+WS_STEP_HOST = 4
+
+EXPORTS = ["ceca_schedule", "ceca_gossip_sgd_step", "ceca_consensus_rounds", "dsgd_logreg_grad",
+           "ceca_workspace_bytes", "ceca_read_status", "ceca_gossip_sgd_step_host", "ceca_status_string"]
+
+
+class Round(ctypes.Structure):
+    """Mirror of ceca_round_t."""
+    _fields_ = [("n", ctypes.c_int32), ("tau", ctypes.c_int32), ("r", ctypes.c_int32),
+                ("delta", ctypes.c_int32), ("n_r", ctypes.c_int32), ("payload", ctypes.c_int32),
+                ("a_num", ctypes.c_int32), ("a_den", ctypes.c_int32),
+                ("b_num", ctypes.c_int32), ("b_den", ctypes.c_int32),
+                ("a", ctypes.c_double), ("b", ctypes.c_double)]
+
+
+class CecaError(RuntimeError):
+    def __init__(self, status, where):
+        self.status = int(status)
+        super().__init__("%s: %s (status %d)" % (where, ceca_status_string(status), status))
+
+
+_lib = None
+
+
+def library_path():
+    return _build.LIB
+
+
+def library():
+    """Loads libceca_b200.so (building it first when it is missing or older than its sources)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    path = _build.build() if (_build.is_stale() and os.environ.get("CECA_NO_BUILD") != "1") else _build.LIB
+    lib = ctypes.CDLL(path)
+    vp, i32, i64, f32 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_float
+    lib.ceca_schedule.argtypes = [i32, i32, i64, ctypes.POINTER(Round), vp, vp]
+    lib.ceca_schedule.restype = ctypes.c_int
+    lib.ceca_gossip_sgd_step.argtypes = [vp, vp, vp, vp, vp, i32, i64, i64, f32, i32, i64, vp]
+    lib.ceca_gossip_sgd_step.restype = ctypes.c_int
+    lib.ceca_consensus_rounds.argtypes = [vp, vp, vp, vp, i32, i64, i64, i32, i64, i32, i32, vp,
+                                          ctypes.c_size_t, vp]
+    lib.ceca_consensus_rounds.restype = ctypes.c_int
+    lib.dsgd_logreg_grad.argtypes = [vp, vp, vp, vp, i64, vp, i32, i32, i64, i64, i32, vp,
+                                     ctypes.c_size_t, vp]
+    lib.dsgd_logreg_grad.restype = ctypes.c_int
+    lib.ceca_workspace_bytes.argtypes = [ctypes.c_int, i32, i32, i64]
+    lib.ceca_workspace_bytes.restype = ctypes.c_size_t
+    lib.ceca_read_status.argtypes = [vp, ctypes.POINTER(i32), vp]
+    lib.ceca_read_status.restype = ctypes.c_int
+    lib.ceca_gossip_sgd_step_host.argtypes = [vp, vp, vp, i32, i64, i64, f32, i32, i64, vp, ctypes.c_size_t]
+    lib.ceca_gossip_sgd_step_host.restype = ctypes.c_int
+    lib.ceca_status_string.argtypes = [ctypes.c_int]
+    lib.ceca_status_string.restype = ctypes.c_char_p
+    _lib = lib
+    return lib
+
+
+def ceca_status_string(status):
+    return library().ceca_status_string(int(status)).decode()
+
+
+def _check(status, where):
+    if status != 0:
+        raise CecaError(status, where)
+
+
+def _ptr(t):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(stream):
+    if stream is None:
+        import torch
+        return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+    return ctypes.c_void_p(getattr(stream, "cuda_stream", stream))
+
+
+def _matrix(t, name, n=None, cuda=True):
+    """(n, d, ld) of a 2-D fp32 tensor whose rows are contiguous."""
+    import torch
+    if t.dtype != torch.float32 or t.dim() != 2 or t.stride(1) != 1:
+        raise ValueError("%s must be a 2-D float32 tensor with unit column stride" % name)
+    if cuda != t.is_cuda:
+        raise ValueError("%s must live in %s memory" % (name, "device" if cuda else "host"))
+    if n is not None and t.shape[0] != n:
+        raise ValueError("%s has the wrong number of rows" % name)
+    return t.shape[0], t.shape[1], t.stride(0) if t.shape[0] > 1 else max(t.stride(0), t.shape[1])
+
+
+def ceca_schedule(n, variant, k, peers=True):
+    """(Round, recv_from, send_to); the peer arrays are int32 numpy arrays (None when peers=False)."""
+    rd = Round()
+    recv = np.empty(max(n, 0), dtype=np.int32) if peers else None
+    send = np.empty(max(n, 0), dtype=np.int32) if peers else None
+    st = library().ceca_schedule(n, variant, k, ctypes.byref(rd),
+                                 recv.ctypes.data if peers else None, send.ctypes.data if peers else None)
+    _check(st, "ceca_schedule")
+    return rd, recv, send
+
+
+def ceca_gossip_sgd_step(X, Y, G, gamma, variant, k, X_out=None, Y_out=None, stream=None):
+    """One DSGD-CECA iteration on device tensors.  Outputs default to in place.  Returns (X_out, Y_out)."""
+    n, d, ld = _matrix(X, "X")
+    X_out = X if X_out is None else X_out
+    if Y_out is None:
+        if Y is None:
+            raise ValueError("Y_out is needed when Y is None")
+        Y_out = Y
+    for t, name in ((Y, "Y"), (G, "G"), (X_out, "X_out"), (Y_out, "Y_out")):
+        if t is not None and _matrix(t, name, n) != (n, d, ld):
+            raise ValueError("%s must have the shape and row stride of X" % name)
+    st = library().ceca_gossip_sgd_step(_ptr(X), _ptr(Y), _ptr(G), _ptr(X_out), _ptr(Y_out), n, d, ld,
+                                        float(gamma), variant, k, _stream(stream))
+    _check(st, "ceca_gossip_sgd_step")
+    return X_out, Y_out
+
+
+def ceca_consensus_rounds(X, Y, variant, k0, rounds, fused, X_out=None, Y_out=None, workspace=None,
+                          want_y=True, stream=None):
+    """`rounds` CECA rounds on device tensors.  Returns (X_out, Y_out); Y_out is None when want_y is false."""
+    n, d, ld = _matrix(X, "X")
+    X_out = X if X_out is None else X_out
+    if want_y and Y_out is None:
+        if Y is None:
+            raise ValueError("Y_out is needed when Y is None and want_y is true")
+        Y_out = Y
+    for t, name in ((Y, "Y"), (X_out, "X_out"), (Y_out, "Y_out")):
+        if t is not None and _matrix(t, name, n) != (n, d, ld):
+            raise ValueError("%s must have the shape and row stride of X" % name)
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    st = library().ceca_consensus_rounds(_ptr(X), _ptr(Y), _ptr(X_out), _ptr(Y_out), n, d, ld, variant, k0,
+                                         rounds, int(bool(fused)), _ptr(workspace), ws_bytes, _stream(stream))
+    _check(st, "ceca_consensus_rounds")
+    return X_out, Y_out
+
+
+def dsgd_logreg_grad(A, labels, X, Y, k, variant, G, workspace, stream=None):
+    """Per-agent logistic gradient at the model iteration k selects; writes G and returns it."""
+    import torch
+    if A.dtype != torch.float32 or A.dim() != 3 or not A.is_contiguous() or not A.is_cuda:
+        raise ValueError("A must be a contiguous 3-D float32 device tensor")
+    n, m, d = A.shape
+    if labels.dtype != torch.float32 or tuple(labels.shape) != (n, m) or not labels.is_contiguous():
+        raise ValueError("labels must be a contiguous float32 [n, m] tensor")
+    _, dx, ld = _matrix(X, "X", n)
+    if dx != d:
+        raise ValueError("X must have d columns")
+    for t, name in ((Y, "Y"), (G, "G")):
+        if t is not None and _matrix(t, name, n) != (n, d, ld):
+            raise ValueError("%s must have the shape and row stride of X" % name)
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    st = library().dsgd_logreg_grad(_ptr(A), _ptr(labels), _ptr(X), _ptr(Y), k, _ptr(G), n, m, d, ld, variant,
+                                    _ptr(workspace), ws_bytes, _stream(stream))
+    _check(st, "dsgd_logreg_grad")
+    return G
+
+
+def ceca_workspace_bytes(kind, n, m, d):
+    return int(library().ceca_workspace_bytes(kind, n, m, d))
+
+
+def ceca_read_status(workspace, stream=None):
+    out = ctypes.c_int32(-1)
+    _check(library().ceca_read_status(_ptr(workspace), ctypes.byref(out), _stream(stream)), "ceca_read_status")
+    return out.value
+
+
+def ceca_gossip_sgd_step_host(X, Y, G, gamma, variant, k, workspace):
+    """The iteration on HOST tensors (updated in place), streamed through a DEVICE workspace."""
+    n, d, ld = _matrix(X, "X", cuda=False)
+    for t, name in ((Y, "Y"), (G, "G")):
+        if t is not None and _matrix(t, name, n, cuda=False) != (n, d, ld):
+            raise ValueError("%s must have the shape and row stride of X" % name)
+    if not workspace.is_cuda:
+        raise ValueError("workspace must be device memory")
+    ws_bytes = workspace.numel() * workspace.element_size()
+    st = library().ceca_gossip_sgd_step_host(_ptr(X), _ptr(Y), _ptr(G), n, d, ld, float(gamma), variant, k,
+                                             _ptr(workspace), ws_bytes)
+    _check(st, "ceca_gossip_sgd_step_host")
+    return X, Y

@@ -1,0 +1,327 @@
+// CECA consensus rounds (Sec. 3.1 "Main recursions", Algorithm 2; Sec. 3.2 for the 1-port pairing).
+//
+// fused = 0: one pass of the step kernel (gamma = 0, no G) per round.
+// fused = 1: one launch.  Each CTA brings an n x W column tile of X (and of Y when the first
+//   round needs it) into shared memory with one TMA tensor load, moves it into registers (a
+//   thread keeps a few rows of one column for the whole run), and runs all rounds on chip: per
+//   round every thread publishes the payload (I or J) of its rows in a shared exchange buffer,
+//   the CTA synchronises, and every thread picks up the value of the row it receives from.  Only
+//   4 bytes per element per round go through shared memory in each direction.  The finished
+//   tiles go back with one TMA tensor store each.  HBM sees X once in and X (and Y) once out,
+//   instead of once per round.
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <cstdint>
+#include <cstring>
+
+#include "ceca.h"
+#include "plan.h"
+
+namespace ceca {
+
+cudaError_t enqueue_step(const Plan &plan, const float *X, const float *Y, const float *G, float *Xo,
+                         float *Yo, int32_t n, int64_t d, int64_t ld, float gamma,
+                         cudaStream_t stream);
+ceca_status_t check_matrix_args(const void *X, const void *X_out, int32_t n, int64_t d, int64_t ld);
+
+constexpr int kMaxFusedRounds = 64;
+constexpr int kMaxFusedRows = 256;   // one TMA box holds at most 256 rows
+constexpr int kTileCols = 32;        // W: columns per CTA tile (128-byte row segments)
+constexpr int kRowGroups = 8;        // Q: a column's rows are dealt round-robin to Q threads
+constexpr int kFusedThreads = kTileCols * kRowGroups;
+constexpr uint32_t kWaitPolls = 1u << 22;  // bounded mbarrier wait (each poll sleeps ~100 ns)
+
+struct FusedRound {
+  int32_t hop;      // 2-port: shift s; 1-port: pairing offset o
+  int32_t payload;  // 0: I is exchanged, 1: J
+  float a, b, one_minus_a, one_minus_b;
+};
+
+struct FusedArgs {
+  int32_t n, rounds, one_port, has_y_in, has_y_out;
+  int32_t *status;
+  FusedRound rd[kMaxFusedRounds];
+};
+
+// ---- PTX wrappers (mbarrier + TMA) ----------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void *p) {
+  return (uint32_t)__cvta_generic_to_shared(p);
+}
+__device__ __forceinline__ void mbar_init(uint64_t *bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t *bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes)
+               : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t phase) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(phase)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait: returns false when the barrier did not flip within the poll budget.
+__device__ __forceinline__ bool mbar_wait_bounded(uint64_t *bar, uint32_t phase, uint32_t polls) {
+  for (uint32_t i = 0; i < polls; ++i) {
+    if (mbar_try_wait(bar, phase)) return true;
+    __nanosleep(64);
+  }
+  return false;
+}
+__device__ __forceinline__ void tma_load_2d(void *dst, const CUtensorMap *map, int32_t x, int32_t y,
+                                            uint64_t *bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(smem_u32(dst)), "l"(map), "r"(x), "r"(y), "r"(smem_u32(bar))
+      : "memory");
+}
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap *map, int32_t x, int32_t y, const void *src) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];"
+               ::"l"(map), "r"(x), "r"(y), "r"(smem_u32(src))
+               : "memory");
+}
+
+// R = rows per thread (compile time), so n <= R * kRowGroups.
+template <int R>
+__global__ void __launch_bounds__(kFusedThreads)
+consensus_fused_kernel(const __grid_constant__ CUtensorMap map_x_in, const __grid_constant__ CUtensorMap map_y_in,
+                       const __grid_constant__ CUtensorMap map_x_out,
+                       const __grid_constant__ CUtensorMap map_y_out, const __grid_constant__ FusedArgs p) {
+  extern __shared__ __align__(128) unsigned char smem_raw[];
+  const int n = p.n;
+  float *tile_a = reinterpret_cast<float *>(smem_raw);            // [n][W]  X tile, then exchange buffer 0
+  float *tile_b = tile_a + (size_t)n * kTileCols;                 // [n][W]  Y tile, then exchange buffer 1
+  __shared__ __align__(8) uint64_t bar;
+
+  const int c = threadIdx.x % kTileCols;
+  const int q = threadIdx.x / kTileCols;
+  const int32_t col0 = (int32_t)blockIdx.x * kTileCols;  // multiple of 32 floats: 16-byte aligned
+
+  if (threadIdx.x == 0) {
+    mbar_init(&bar, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    const uint32_t tile_bytes = (uint32_t)n * kTileCols * sizeof(float);
+    mbar_expect_tx(&bar, p.has_y_in ? 2 * tile_bytes : tile_bytes);
+    tma_load_2d(tile_a, &map_x_in, col0, 0, &bar);
+    if (p.has_y_in) tma_load_2d(tile_b, &map_y_in, col0, 0, &bar);
+  }
+  const bool landed = mbar_wait_bounded(&bar, 0, kWaitPolls);
+  if (!__syncthreads_and(landed)) {  // one decision for the whole CTA
+    // The transfer never arrived: flag it, give it one more bounded chance to land (so that
+    // it cannot write into shared memory of a finished CTA), and give up without storing.
+    if (threadIdx.x == 0) atomicExch(p.status, 1);
+    mbar_wait_bounded(&bar, 0, kWaitPolls);
+    return;
+  }
+
+  float I[R], J[R];
+#pragma unroll
+  for (int t = 0; t < R; ++t) {
+    const int i = q + t * kRowGroups;
+    I[t] = i < n ? tile_a[i * kTileCols + c] : 0.f;
+    J[t] = (i < n && p.has_y_in) ? tile_b[i * kTileCols + c] : 0.f;
+  }
+  __syncthreads();  // both tiles are now free to serve as exchange buffers
+
+  for (int rnd = 0; rnd < p.rounds; ++rnd) {
+    const FusedRound rd = p.rd[rnd];
+    float *buf = (rnd & 1) ? tile_b : tile_a;
+#pragma unroll
+    for (int t = 0; t < R; ++t) {
+      const int i = q + t * kRowGroups;
+      if (i < n) buf[i * kTileCols + c] = rd.payload ? J[t] : I[t];
+    }
+    __syncthreads();
+#pragma unroll
+    for (int t = 0; t < R; ++t) {
+      const int i = q + t * kRowGroups;
+      if (i < n) {
+        int src;
+        if (p.one_port && !(i & 1)) { src = i + rd.hop; if (src >= n) src -= n; }
+        else                        { src = i - rd.hop; if (src < 0) src += n; }
+        const float recv = buf[src * kTileCols + c];
+        I[t] = fmaf(rd.a, I[t], rd.one_minus_a * recv);
+        J[t] = fmaf(rd.b, J[t], rd.one_minus_b * recv);
+      }
+    }
+    // no second barrier: the next round writes the other buffer, and a thread can only start
+    // the round after that once everybody has passed the next round's barrier.
+  }
+  __syncthreads();
+
+#pragma unroll
+  for (int t = 0; t < R; ++t) {
+    const int i = q + t * kRowGroups;
+    if (i < n) {
+      tile_a[i * kTileCols + c] = I[t];
+      if (p.has_y_out) tile_b[i * kTileCols + c] = J[t];
+    }
+  }
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic writes -> visible to TMA
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    tma_store_2d(&map_x_out, col0, 0, tile_a);
+    if (p.has_y_out) tma_store_2d(&map_y_out, col0, 0, tile_b);
+    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+    asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");  // smem must outlive the reads
+  }
+}
+
+// ---- host side ------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_tiled_fn() {
+  static EncodeTiledFn fn = []() -> EncodeTiledFn {
+    void *sym = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &q) != cudaSuccess ||
+        q != cudaDriverEntryPointSuccess)
+      return nullptr;
+    return reinterpret_cast<EncodeTiledFn>(sym);
+  }();
+  return fn;
+}
+
+// An n x d fp32 matrix with row pitch ld, boxed as n rows x kTileCols columns.
+static bool make_map(CUtensorMap *map, const float *base, int32_t n, int64_t d, int64_t ld) {
+  EncodeTiledFn enc = encode_tiled_fn();
+  if (!enc) return false;
+  const cuuint64_t dims[2] = {(cuuint64_t)d, (cuuint64_t)n};
+  const cuuint64_t strides[1] = {(cuuint64_t)ld * sizeof(float)};
+  const cuuint32_t box[2] = {(cuuint32_t)kTileCols, (cuuint32_t)n};
+  const cuuint32_t elem[2] = {1, 1};
+  return enc(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float *>(base), dims, strides, box, elem,
+             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int R>
+static cudaError_t launch_fused(const CUtensorMap &mxi, const CUtensorMap &myi, const CUtensorMap &mxo,
+                                const CUtensorMap &myo, const FusedArgs &args, int64_t d,
+                                cudaStream_t stream) {
+  const size_t smem = 2 * (size_t)args.n * kTileCols * sizeof(float);
+  cudaError_t e = cudaFuncSetAttribute(consensus_fused_kernel<R>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       (int)smem);
+  if (e != cudaSuccess) return e;
+  const int64_t tiles = (d + kTileCols - 1) / kTileCols;
+  consensus_fused_kernel<R><<<(unsigned)tiles, kFusedThreads, smem, stream>>>(mxi, myi, mxo, myo, args);
+  return cudaGetLastError();
+}
+
+static inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+static ceca_status_t consensus_fused(const float *X, const float *Y, float *Xo, float *Yo, int32_t n, int64_t d,
+                                     int64_t ld, ceca_variant_t variant, int64_t k0, int32_t rounds,
+                                     void *workspace, size_t workspace_bytes, cudaStream_t stream) {
+  if (n > kMaxFusedRows || rounds > kMaxFusedRounds || ld >= ((int64_t)1 << 32) || d > 0x7fffffffLL)
+    return CECA_ERR_UNSUPPORTED;
+  if (!workspace || workspace_bytes < sizeof(int32_t) || !aligned16(workspace)) return CECA_ERR_WORKSPACE;
+  FusedArgs args;
+  std::memset(&args, 0, sizeof(args));
+  args.n = n; args.rounds = rounds; args.one_port = (variant == CECA_1P);
+  args.status = static_cast<int32_t *>(workspace);
+  bool first_needs_y = false;
+  for (int32_t t = 0; t < rounds; ++t) {
+    Plan plan;
+    ceca_status_t st = make_plan(n, variant, k0 + t, &plan);
+    if (st != CECA_OK) return st;
+    if (t == 0) first_needs_y = plan.reads_y;
+    FusedRound &r = args.rd[t];
+    r.hop = plan.walk.hop;  // 2-port: the shift; 1-port: the pairing offset
+    r.payload = plan.rd.payload;
+    r.a = plan.a; r.b = plan.b; r.one_minus_a = plan.one_minus_a; r.one_minus_b = plan.one_minus_b;
+  }
+  if (first_needs_y && !Y) return CECA_ERR_INVALID_ARG;
+  args.has_y_in = (Y != nullptr && first_needs_y) ? 1 : 0;
+  args.has_y_out = Yo ? 1 : 0;
+  if ((ld % 4) != 0 || !aligned16(X) || !aligned16(Xo) || (args.has_y_in && !aligned16(Y)) ||
+      (Yo && !aligned16(Yo)))
+    return CECA_ERR_ALIGNMENT;
+
+  CUtensorMap mxi, myi, mxo, myo;
+  if (!make_map(&mxi, X, n, d, ld) || !make_map(&mxo, Xo, n, d, ld)) return CECA_ERR_CUDA;
+  if (!make_map(&myi, args.has_y_in ? Y : X, n, d, ld)) return CECA_ERR_CUDA;
+  if (!make_map(&myo, Yo ? Yo : Xo, n, d, ld)) return CECA_ERR_CUDA;
+
+  const int rows_per_thread = (n + kRowGroups - 1) / kRowGroups;
+  cudaError_t e;
+  if (rows_per_thread <= 4)       e = launch_fused<4>(mxi, myi, mxo, myo, args, d, stream);
+  else if (rows_per_thread <= 8)  e = launch_fused<8>(mxi, myi, mxo, myo, args, d, stream);
+  else if (rows_per_thread <= 13) e = launch_fused<13>(mxi, myi, mxo, myo, args, d, stream);
+  else if (rows_per_thread <= 16) e = launch_fused<16>(mxi, myi, mxo, myo, args, d, stream);
+  else if (rows_per_thread <= 24) e = launch_fused<24>(mxi, myi, mxo, myo, args, d, stream);
+  else                            e = launch_fused<32>(mxi, myi, mxo, myo, args, d, stream);
+  return e == cudaSuccess ? CECA_OK : CECA_ERR_CUDA;
+}
+
+}  // namespace ceca
+
+extern "C" ceca_status_t ceca_consensus_rounds(const float *X, const float *Y, float *X_out, float *Y_out,
+                                               int32_t n, int64_t d, int64_t ld, ceca_variant_t variant,
+                                               int64_t k0, int32_t rounds, int32_t fused, void *workspace,
+                                               size_t workspace_bytes, void *stream_) {
+  using namespace ceca;
+  ceca_status_t st = check_matrix_args(X, X_out, n, d, ld);
+  if (st != CECA_OK) return st;
+  if (rounds < 0 || k0 < 0) return CECA_ERR_INVALID_ARG;
+  if (X_out == Y_out || (const float *)X_out == Y || (Y_out && (const float *)Y_out == X))
+    return CECA_ERR_UNSUPPORTED;
+  Plan first;
+  st = make_plan(n, variant, k0, &first);  // also validates the variant / parity of n
+  if (st != CECA_OK) return st;
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+
+  if (rounds == 0 || n == 1) {  // nothing to mix: the result is a copy of the input
+    cudaError_t e = cudaSuccess;
+    if (X_out != X)
+      e = cudaMemcpy2DAsync(X_out, ld * sizeof(float), X, ld * sizeof(float), d * sizeof(float), n,
+                            cudaMemcpyDeviceToDevice, stream);
+    if (e == cudaSuccess && Y_out && Y && Y_out != Y)
+      e = cudaMemcpy2DAsync(Y_out, ld * sizeof(float), Y, ld * sizeof(float), d * sizeof(float), n,
+                            cudaMemcpyDeviceToDevice, stream);
+    if (Y_out && !Y) return CECA_ERR_INVALID_ARG;
+    return e == cudaSuccess ? CECA_OK : CECA_ERR_CUDA;
+  }
+
+  if (fused)
+    return consensus_fused(X, Y, X_out, Y_out, n, d, ld, variant, k0, rounds, workspace, workspace_bytes,
+                           stream);
+
+  if (!Y && first.reads_y) return CECA_ERR_INVALID_ARG;
+  float *y_work = Y_out;
+  if (!y_work) {  // the caller does not want Y back: keep it in the workspace
+    if (!workspace || workspace_bytes < (size_t)n * (size_t)ld * sizeof(float)) return CECA_ERR_WORKSPACE;
+    y_work = static_cast<float *>(workspace);
+    if ((const float *)y_work == X || (const float *)y_work == Y || y_work == X_out) return CECA_ERR_UNSUPPORTED;
+  }
+  const float *x_in = X, *y_in = Y;
+  for (int32_t t = 0; t < rounds; ++t) {
+    Plan plan;
+    st = make_plan(n, variant, k0 + t, &plan);
+    if (st != CECA_OK) return st;
+    cudaError_t e = enqueue_step(plan, x_in, y_in, nullptr, X_out, y_work, n, d, ld, 0.f, stream);
+    if (e != cudaSuccess) return CECA_ERR_CUDA;
+    x_in = X_out; y_in = y_work;  // later rounds run in place on the outputs
+  }
+  return CECA_OK;
+}
+
+extern "C" ceca_status_t ceca_read_status(const void *workspace, int32_t *status_out, void *stream) {
+  if (!workspace || !status_out) return CECA_ERR_INVALID_ARG;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (cudaMemcpyAsync(status_out, workspace, sizeof(int32_t), cudaMemcpyDeviceToHost, s) != cudaSuccess)
+    return CECA_ERR_CUDA;
+  return cudaStreamSynchronize(s) == cudaSuccess ? CECA_OK : CECA_ERR_CUDA;
+}

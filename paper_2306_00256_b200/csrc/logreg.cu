@@ -1,0 +1,237 @@
+// Per-agent logistic-regression gradient (the e^(k) of Algorithm 1 for the synthetic
+// classification workloads; the loss itself is not from the paper):
+//   G[i, :] = -(1/m) sum_s l_s sigma(-l_s <a_s, z_i>) a_s,   z = X if delta_r = 1 else Y.
+//
+// Main path (d a multiple of 4, d <= 8192, 16-byte aligned rows): A is read exactly once.  A CTA
+// takes one agent and a block of its samples; each thread keeps its slice of z_i and of the
+// running gradient in registers, loads its slice of four sample rows, the CTA reduces the four
+// inner products (warp shuffles, then a fixed-order sum over the warps through shared memory),
+// every thread turns them into the four coefficients and adds coefficient * row slice to its
+// gradient slice.  Per-CTA partial gradients go to the workspace and a second kernel adds them in
+// a fixed order, so the result does not change from run to run.  Not a dense contraction worth
+// tensor cores: two matrix-vector products per agent, bound by reading A from HBM.
+//
+// Fallback (any d, any alignment): coefficients first (one warp per sample), then a column-wise
+// accumulation; A is read twice.
+#include <cuda_runtime.h>
+
+#include <cstdint>
+
+#include "ceca.h"
+#include "plan.h"
+
+namespace ceca {
+
+constexpr int kLrThreads = 256;
+constexpr int kLrWarps = kLrThreads / 32;
+constexpr int kLrSamples = 4;        // sample rows in flight per thread
+constexpr int kLrMaxVpt = 8;         // float4 column groups per thread -> d <= 256*4*8 = 8192
+constexpr int kLrTargetCtas = 148 * 12;
+
+static inline int32_t logreg_sample_blocks(int32_t n, int32_t m) {
+  int64_t p = (kLrTargetCtas + n - 1) / n;
+  const int64_t most = (m + 4 * kLrSamples - 1) / (4 * kLrSamples);  // at least 16 samples per block
+  if (p > most) p = most;
+  if (p < 1) p = 1;
+  return (int32_t)p;
+}
+
+struct LogregArgs {
+  const float *A, *labels, *Z;
+  float *partial;   // [n][P][d]
+  int64_t d, ld;
+  int32_t n, m, P, samples_per_block;
+  float inv_m;
+};
+
+__device__ __forceinline__ float dot4(float4 a, float4 b) {
+  return fmaf(a.x, b.x, fmaf(a.y, b.y, fmaf(a.z, b.z, a.w * b.w)));
+}
+
+template <int VPT>
+__global__ void __launch_bounds__(kLrThreads) logreg_fused_kernel(const LogregArgs p) {
+  __shared__ float4 red[2][kLrWarps];
+  const int i = blockIdx.y;
+  const int blk = blockIdx.x;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int64_t d4 = p.d >> 2;
+  const int s_begin = blk * p.samples_per_block;
+  const int s_end = min(p.m, s_begin + p.samples_per_block);
+
+  float4 z[VPT], acc[VPT];
+  bool valid[VPT];
+#pragma unroll
+  for (int j = 0; j < VPT; ++j) {
+    const int64_t cg = threadIdx.x + (int64_t)j * kLrThreads;
+    valid[j] = cg < d4;
+    z[j] = valid[j] ? *reinterpret_cast<const float4 *>(p.Z + (int64_t)i * p.ld + cg * 4)
+                    : make_float4(0.f, 0.f, 0.f, 0.f);
+    acc[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+  }
+  const float *a_agent = p.A + (int64_t)i * p.m * p.d;
+  const float *l_agent = p.labels + (int64_t)i * p.m;
+
+  int buf = 0;
+  for (int s = s_begin; s < s_end; s += kLrSamples) {
+    float4 a[kLrSamples][VPT];
+    float dot[kLrSamples];
+#pragma unroll
+    for (int jj = 0; jj < kLrSamples; ++jj) {
+      const bool live = s + jj < s_end;
+      const float *row = a_agent + (int64_t)(s + jj) * p.d;
+#pragma unroll
+      for (int j = 0; j < VPT; ++j) {
+        const int64_t cg = threadIdx.x + (int64_t)j * kLrThreads;
+        a[jj][j] = (live && valid[j]) ? __ldcs(reinterpret_cast<const float4 *>(row + cg * 4))
+                                      : make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+    }
+#pragma unroll
+    for (int jj = 0; jj < kLrSamples; ++jj) {
+      float t = 0.f;
+#pragma unroll
+      for (int j = 0; j < VPT; ++j) t += dot4(a[jj][j], z[j]);
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
+      dot[jj] = t;
+    }
+    if (lane == 0) red[buf][warp] = make_float4(dot[0], dot[1], dot[2], dot[3]);
+    __syncthreads();
+    float4 tot = red[buf][0];
+#pragma unroll
+    for (int w = 1; w < kLrWarps; ++w) {
+      const float4 v = red[buf][w];
+      tot.x += v.x; tot.y += v.y; tot.z += v.z; tot.w += v.w;
+    }
+    buf ^= 1;  // the other buffer is free: everybody passed the barrier above after reading it
+    const float margin[kLrSamples] = {tot.x, tot.y, tot.z, tot.w};
+#pragma unroll
+    for (int jj = 0; jj < kLrSamples; ++jj) {
+      float coef = 0.f;
+      if (s + jj < s_end) {
+        const float l = __ldg(l_agent + s + jj);
+        coef = -l * p.inv_m / (1.f + expf(l * margin[jj]));  // -l sigma(-l t) / m
+      }
+#pragma unroll
+      for (int j = 0; j < VPT; ++j) {
+        acc[j].x = fmaf(coef, a[jj][j].x, acc[j].x);
+        acc[j].y = fmaf(coef, a[jj][j].y, acc[j].y);
+        acc[j].z = fmaf(coef, a[jj][j].z, acc[j].z);
+        acc[j].w = fmaf(coef, a[jj][j].w, acc[j].w);
+      }
+    }
+  }
+  float *out = p.partial + ((int64_t)i * p.P + blk) * p.d;
+#pragma unroll
+  for (int j = 0; j < VPT; ++j) {
+    const int64_t cg = threadIdx.x + (int64_t)j * kLrThreads;
+    if (valid[j]) *reinterpret_cast<float4 *>(out + cg * 4) = acc[j];
+  }
+}
+
+// G[i, c..c+3] = sum over the P partials, in block order.
+__global__ void __launch_bounds__(256) logreg_reduce_kernel(const float *partial, float *G, int32_t n, int32_t P,
+                                                            int64_t d, int64_t ld) {
+  const int64_t d4 = d >> 2;
+  const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= (int64_t)n * d4) return;
+  const int64_t i = idx / d4, cg = idx - i * d4;
+  const float *src = partial + i * P * d + cg * 4;
+  float4 s = *reinterpret_cast<const float4 *>(src);
+  for (int32_t b = 1; b < P; ++b) {
+    const float4 v = *reinterpret_cast<const float4 *>(src + (int64_t)b * d);
+    s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
+  }
+  *reinterpret_cast<float4 *>(G + i * ld + cg * 4) = s;
+}
+
+// ---- fallback: any d, any alignment ---------------------------------------------------------
+__global__ void __launch_bounds__(256) logreg_coef_kernel(const float *A, const float *labels, const float *Z,
+                                                          float *coef, int32_t n, int32_t m, int64_t d, int64_t ld,
+                                                          float inv_m) {
+  const int64_t sample = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;  // one warp per sample
+  const int lane = threadIdx.x & 31;
+  if (sample >= (int64_t)n * m) return;
+  const int64_t i = sample / m;
+  const float *row = A + sample * d;
+  const float *z = Z + i * ld;
+  float t = 0.f;
+  for (int64_t c = lane; c < d; c += 32) t = fmaf(row[c], z[c], t);
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
+  if (lane == 0) {
+    const float l = labels[sample];
+    coef[sample] = -l * inv_m / (1.f + expf(l * t));
+  }
+}
+
+__global__ void __launch_bounds__(256) logreg_accum_kernel(const float *A, const float *coef, float *G, int32_t n,
+                                                           int32_t m, int64_t d, int64_t ld) {
+  const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= (int64_t)n * d) return;
+  const int64_t i = idx / d, c = idx - i * d;
+  const float *col = A + i * m * d + c;
+  const float *cf = coef + i * m;
+  float g = 0.f;
+  for (int32_t s = 0; s < m; ++s) g = fmaf(cf[s], col[(int64_t)s * d], g);
+  G[i * ld + c] = g;
+}
+
+static inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+size_t logreg_workspace_bytes(int32_t n, int32_t m, int64_t d) {
+  const size_t partial = (size_t)n * (size_t)logreg_sample_blocks(n, m) * (size_t)d * sizeof(float);
+  const size_t coef = (size_t)n * (size_t)m * sizeof(float);
+  return ((partial + 255) / 256) * 256 + ((coef + 255) / 256) * 256;
+}
+
+}  // namespace ceca
+
+extern "C" ceca_status_t dsgd_logreg_grad(const float *A, const float *labels, const float *X, const float *Y,
+                                          int64_t k, float *G, int32_t n, int32_t m, int64_t d, int64_t ld,
+                                          ceca_variant_t variant, void *workspace, size_t workspace_bytes,
+                                          void *stream_) {
+  using namespace ceca;
+  if (!A || !labels || !X || !G || n < 1 || m < 1 || d < 1 || ld < d) return CECA_ERR_INVALID_ARG;
+  Plan plan;
+  ceca_status_t st = make_plan(n, variant, k, &plan);
+  if (st != CECA_OK) return st;
+  const float *Z = plan.rd.payload ? Y : X;
+  if (!Z) return CECA_ERR_INVALID_ARG;
+  if (!workspace || workspace_bytes < logreg_workspace_bytes(n, m, d) || !aligned16(workspace))
+    return CECA_ERR_WORKSPACE;
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  const float inv_m = (float)(1.0 / (double)m);
+  const int32_t P = logreg_sample_blocks(n, m);
+  float *partial = static_cast<float *>(workspace);
+  const size_t partial_bytes = (((size_t)n * P * d * sizeof(float) + 255) / 256) * 256;
+  float *coef = reinterpret_cast<float *>(static_cast<char *>(workspace) + partial_bytes);
+
+  const bool fast = (d % 4 == 0) && (ld % 4 == 0) && d <= (int64_t)kLrThreads * 4 * kLrMaxVpt && aligned16(A) &&
+                    aligned16(Z) && aligned16(G) && n <= 65535;
+  if (fast) {
+    LogregArgs a;
+    a.A = A; a.labels = labels; a.Z = Z; a.partial = partial;
+    a.d = d; a.ld = ld; a.n = n; a.m = m; a.P = P;
+    a.samples_per_block = (m + P - 1) / P;
+    a.inv_m = inv_m;
+    const dim3 grid((unsigned)P, (unsigned)n);
+    const int64_t groups = (d / 4 + kLrThreads - 1) / kLrThreads;
+    if (groups <= 1)      logreg_fused_kernel<1><<<grid, kLrThreads, 0, stream>>>(a);
+    else if (groups <= 2) logreg_fused_kernel<2><<<grid, kLrThreads, 0, stream>>>(a);
+    else if (groups <= 4) logreg_fused_kernel<4><<<grid, kLrThreads, 0, stream>>>(a);
+    else                  logreg_fused_kernel<8><<<grid, kLrThreads, 0, stream>>>(a);
+    if (cudaGetLastError() != cudaSuccess) return CECA_ERR_CUDA;
+    const int64_t work = (int64_t)n * (d / 4);
+    logreg_reduce_kernel<<<(unsigned)((work + 255) / 256), 256, 0, stream>>>(partial, G, n, P, d, ld);
+    return cudaGetLastError() == cudaSuccess ? CECA_OK : CECA_ERR_CUDA;
+  }
+  const int64_t warps = (int64_t)n * m;
+  const int64_t blocks1 = (warps * 32 + 255) / 256;
+  const int64_t blocks2 = ((int64_t)n * d + 255) / 256;
+  if (blocks1 > 0x7fffffffLL || blocks2 > 0x7fffffffLL) return CECA_ERR_UNSUPPORTED;
+  logreg_coef_kernel<<<(unsigned)blocks1, 256, 0, stream>>>(A, labels, Z, coef, n, m, d, ld, inv_m);
+  if (cudaGetLastError() != cudaSuccess) return CECA_ERR_CUDA;
+  logreg_accum_kernel<<<(unsigned)blocks2, 256, 0, stream>>>(A, coef, G, n, m, d, ld);
+  return cudaGetLastError() == cudaSuccess ? CECA_OK : CECA_ERR_CUDA;
+}

@@ -1,0 +1,392 @@
+"""GPU parity: the CUDA library against the fp64 oracle, element by element, on the same seeded
+fp32 inputs.  Every call goes through the C ABI (via the ctypes binding).
+
+Tolerances (fp32 arithmetic against fp64):
+  * one step / one round: max|delta| <= 2e-6 * scale, scale = max(|X|, |Y|, |gamma| |G|) of the inputs
+    (the stated 2e-6 * max|X| bound, with the other operands included so that X0 = 0 is testable);
+  * r rounds: r times that;
+  * after tau aligned rounds the consensus deviation ||X - 1 xbar^T||_F / ||X||_F <= 1e-5;
+  * logistic gradient: 8 sqrt(d) 2^-24 max|G| + 1e-7 (a length-d fp32 dot product feeding a
+    1/4-Lipschitz sigmoid, then a length-m fp32 sum).
+Schedules and peer indices are compared bit for bit in the CPU tests.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2306_00256_b200 as ceca
+import synthetic_inputs as synth
+
+pytestmark = pytest.mark.gpu
+
+DEV = "cuda:0"
+STEP_TOL = 2e-6
+
+
+def _np(t):
+    return t.detach().cpu().numpy()
+
+
+def _scale(gamma, *tensors):
+    vals = []
+    for t, w in tensors:
+        if t is not None:
+            vals.append(float(t.abs().max()) * w)
+    return max(vals + [1e-30])
+
+
+def _padded(n, d, ld, offset=0):
+    """A [n, d] view with row stride ld, starting `offset` floats into a fresh buffer."""
+    buf = torch.full((n * ld + offset + 8,), float("nan"), dtype=torch.float32, device=DEV)
+    return buf[offset:offset + n * ld].view(n, ld)[:, :d], buf
+
+
+def _put(src, ld=None, offset=0):
+    n, d = src.shape
+    view, buf = _padded(n, d, ld or d, offset)
+    view.copy_(src)
+    return view, buf
+
+
+def _variants(n):
+    return [ceca.CECA_2P] if (n % 2 and n > 1) else [ceca.CECA_2P, ceca.CECA_1P]
+
+
+def _tau(n):
+    return max(oracle.round_info(n, 0).tau, 1)
+
+
+# --------------------------------------------------------------------------------------------
+# fused SGD step + gossip round
+# --------------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("n", [1, 2, 3, 5, 6, 24, 63, 64, 97, 100])
+@pytest.mark.parametrize("d", [1, 3, 4, 5, 1023, 4100, 70001])
+def test_step_matches_oracle_every_round(n, d):
+    x, y, g = synth.step_inputs(n, d, seed=n * 1000 + d, x_std=1.0, g_std=1.0, same_xy=False)
+    gamma = 0.1
+    for variant in _variants(n):
+        for k in list(range(_tau(n))) + [2**40 + 1]:
+            X, Y, G = x.to(DEV), y.to(DEV), g.to(DEV)
+            Xo, Yo = torch.empty_like(X), torch.empty_like(Y)
+            ceca.ceca_gossip_sgd_step(X, Y, G, gamma, variant, k, X_out=Xo, Y_out=Yo)
+            want_x, want_y = oracle.step(_np(x), _np(y), _np(g), np.float32(gamma), variant, k)
+            tol = STEP_TOL * _scale(gamma, (x, 1), (y, 1), (g, gamma))
+            assert np.abs(_np(Xo) - want_x).max() <= tol, (n, d, variant, k)
+            assert np.abs(_np(Yo) - want_y).max() <= tol, (n, d, variant, k)
+            # inputs untouched by the out-of-place call
+            assert torch.equal(X.cpu(), x) and torch.equal(Y.cpu(), y) and torch.equal(G.cpu(), g)
+            # in place gives the same bits
+            ceca.ceca_gossip_sgd_step(X, Y, G, gamma, variant, k)
+            assert torch.equal(X, Xo) and torch.equal(Y, Yo)
+
+
+@pytest.mark.parametrize("n,d,ld,offset", [(6, 37, 40, 0), (6, 37, 41, 0), (24, 1000, 1024, 4), (24, 1000, 1024, 1),
+                                           (97, 513, 517, 3), (100, 4096, 4100, 0)])
+def test_step_padded_rows_and_unaligned_bases(n, d, ld, offset):
+    x, y, g = synth.step_inputs(n, d, seed=7, x_std=1.0, g_std=0.5, same_xy=False)
+    gamma = 0.25
+    for variant in _variants(n):
+        for k in range(_tau(n)):
+            (X, xb), (Y, yb), (G, gb) = _put(x.to(DEV), ld, offset), _put(y.to(DEV), ld, offset), _put(g.to(DEV), ld, offset)
+            (Xo, xob), (Yo, yob) = _padded(n, d, ld, offset), _padded(n, d, ld, offset)
+            ceca.ceca_gossip_sgd_step(X, Y, G, gamma, variant, k, X_out=Xo, Y_out=Yo)
+            want_x, want_y = oracle.step(_np(x), _np(y), _np(g), np.float32(gamma), variant, k)
+            tol = STEP_TOL * _scale(gamma, (x, 1), (y, 1), (g, gamma))
+            assert np.abs(_np(Xo) - want_x).max() <= tol
+            assert np.abs(_np(Yo) - want_y).max() <= tol
+            # the padding between rows (and around the buffer) is never written
+            if ld > d:
+                assert torch.isnan(xob[offset:offset + n * ld].view(n, ld)[:, d:]).all()
+                assert torch.isnan(yob[offset:offset + n * ld].view(n, ld)[:, d:]).all()
+            assert torch.isnan(xob[:offset]).all() and torch.isnan(xob[offset + n * ld:]).all()
+
+
+def test_step_without_gradient_is_a_ceca_round_and_y_may_be_absent_in_round_zero():
+    n, d = 24, 2051
+    x, y, _ = synth.step_inputs(n, d, seed=3, x_std=1.0, same_xy=False)
+    for variant in _variants(n):
+        for k in range(_tau(n)):
+            X, Y = x.to(DEV), y.to(DEV)
+            Xo, Yo = torch.empty_like(X), torch.empty_like(Y)
+            ceca.ceca_gossip_sgd_step(X, Y, None, 0.3, variant, k, X_out=Xo, Y_out=Yo)
+            want_x, want_y = oracle.step(_np(x), _np(y), None, 0.0, variant, k)
+            tol = STEP_TOL * _scale(0, (x, 1), (y, 1))
+            assert np.abs(_np(Xo) - want_x).max() <= tol and np.abs(_np(Yo) - want_y).max() <= tol
+        Xo2, Yo2 = torch.empty_like(X), torch.empty_like(Y)
+        ceca.ceca_gossip_sgd_step(x.to(DEV), None, None, 0.0, variant, 0, X_out=Xo2, Y_out=Yo2)
+        want_x, want_y = oracle.step(_np(x), np.zeros_like(_np(x)), None, 0.0, variant, 0)
+        assert np.abs(_np(Xo2) - want_x).max() <= tol and np.abs(_np(Yo2) - want_y).max() <= tol
+        with pytest.raises(ceca.CecaError):
+            ceca.ceca_gossip_sgd_step(x.to(DEV), None, None, 0.0, variant, 1, X_out=Xo2, Y_out=Yo2)
+
+
+@pytest.mark.parametrize("n,variant", [(5, ceca.CECA_2P), (6, ceca.CECA_1P), (63, ceca.CECA_2P), (64, ceca.CECA_1P)])
+def test_mean_lemma_and_resume_on_gpu(n, variant):
+    """Lemma "relation between averaged variables": with x0 = y0 the mean takes a plain SGD step.
+    Also: stopping and restarting from (X, Y, k) gives the same bits as running straight through."""
+    d = 3001
+    x, y, _ = synth.step_inputs(n, d, seed=11, x_std=1.0)
+    X, Y = x.to(DEV), y.to(DEV)
+    gamma = 0.05
+    tau = _tau(n)
+    snap = None
+    for k in range(2 * tau + 3):
+        G = synth.gradient_inputs(n, d, k, g_std=1.0, device=DEV)
+        mean_before = X.double().mean(0)
+        ceca.ceca_gossip_sgd_step(X, Y, G, gamma, variant, k)
+        want = mean_before - gamma * G.double().mean(0)
+        assert (X.double().mean(0) - want).abs().max() <= 5e-6
+        assert (Y.double().mean(0) - want).abs().max() <= 5e-6
+        if k == tau:
+            snap = (X.clone(), Y.clone())
+    X2, Y2 = snap
+    for k in range(tau + 1, 2 * tau + 3):
+        G = synth.gradient_inputs(n, d, k, g_std=1.0, device=DEV)
+        ceca.ceca_gossip_sgd_step(X2, Y2, G, gamma, variant, k)
+    assert torch.equal(X, X2) and torch.equal(Y, Y2)
+
+
+# --------------------------------------------------------------------------------------------
+# consensus rounds: one launch per round, and the fused TMA kernel
+# --------------------------------------------------------------------------------------------
+
+def _fused_ws():
+    return torch.zeros(64, dtype=torch.int32, device=DEV)
+
+
+@pytest.mark.parametrize("fused", [0, 1])
+@pytest.mark.parametrize("n", [2, 5, 6, 24, 63, 97, 100, 128, 130, 200, 256])
+@pytest.mark.parametrize("d", [32, 1000, 4100])
+def test_consensus_matches_oracle_and_reaches_the_mean(fused, n, d):
+    x = synth.consensus_inputs(n, d, seed=n + d)
+    y0 = synth.consensus_inputs(n, d, seed=n + d + 1, offset_rows=False)
+    tau = _tau(n)
+    for variant in _variants(n):
+        for k0, rounds in [(0, tau), (0, tau + 1), (0, 1), (1 % tau, 2 * tau + 3), (5 * tau, tau)]:
+            X, Y = x.to(DEV), y0.to(DEV)
+            Xo, Yo = torch.empty_like(X), torch.empty_like(Y)
+            ws = _fused_ws()
+            ceca.ceca_consensus_rounds(X, Y, variant, k0, rounds, fused, X_out=Xo, Y_out=Yo, workspace=ws)
+            assert ceca.ceca_read_status(ws) == 0
+            want_x, want_y = oracle.consensus(_np(x), _np(y0), variant, k0, rounds)
+            tol = STEP_TOL * rounds * _scale(0, (x, 1), (y0, 1))
+            assert np.abs(_np(Xo) - want_x).max() <= tol, (n, d, variant, k0, rounds)
+            assert np.abs(_np(Yo) - want_y).max() <= tol, (n, d, variant, k0, rounds)
+            assert torch.equal(X.cpu(), x) and torch.equal(Y.cpu(), y0)
+            if k0 % tau == 0 and rounds >= tau:
+                xd = Xo.double()
+                mean = x.double().mean(0).to(DEV)
+                dev = (xd - mean).norm() / xd.norm()
+                assert float(dev) <= 1e-5
+                if rounds == tau:  # Y holds the mean of the other agents
+                    loo = (x.double().sum(0, keepdim=True) - x.double()) / (n - 1)
+                    assert (Yo.double().cpu() - loo).abs().max() <= tol
+            # in place gives the same bits
+            ceca.ceca_consensus_rounds(X, Y, variant, k0, rounds, fused, workspace=ws)
+            assert torch.equal(X, Xo) and torch.equal(Y, Yo)
+
+
+@pytest.mark.parametrize("fused", [0, 1])
+def test_consensus_optional_y(fused):
+    n, d = 97, 1000
+    x = synth.consensus_inputs(n, d, seed=5)
+    tau = _tau(n)
+    X = x.to(DEV)
+    want_x, want_y = oracle.consensus(_np(x), np.zeros((n, d)), ceca.CECA_2P, 0, tau)
+    tol = STEP_TOL * tau * float(x.abs().max())
+    # no Y in (round 0 ignores it), Y out wanted
+    Xo, Yo = torch.empty_like(X), torch.empty_like(X)
+    ws = _fused_ws()
+    ceca.ceca_consensus_rounds(X, None, ceca.CECA_2P, 0, tau, fused, X_out=Xo, Y_out=Yo, workspace=ws)
+    assert np.abs(_np(Xo) - want_x).max() <= tol and np.abs(_np(Yo) - want_y).max() <= tol
+    # no Y at all: fused needs only its status word, unfused keeps Y in the workspace
+    Xo2 = torch.empty_like(X)
+    if fused:
+        ws2 = _fused_ws()
+    else:
+        ws2 = torch.empty(ceca.ceca_workspace_bytes(ceca.WS_CONSENSUS_UNFUSED, n, 0, d) // 4, dtype=torch.float32, device=DEV)
+    ceca.ceca_consensus_rounds(X, None, ceca.CECA_2P, 0, tau, fused, X_out=Xo2, workspace=ws2, want_y=False)
+    assert torch.equal(Xo2, Xo)
+    # zero rounds and a single agent are copies
+    Xc, Yc = torch.empty_like(X), torch.empty_like(X)
+    ceca.ceca_consensus_rounds(X, X.clone(), ceca.CECA_2P, 3, 0, fused, X_out=Xc, Y_out=Yc, workspace=ws)
+    assert torch.equal(Xc, X) and torch.equal(Yc, X)
+    one = x[:1].to(DEV).contiguous()
+    oc, yc = torch.empty_like(one), torch.empty_like(one)
+    ceca.ceca_consensus_rounds(one, one.clone(), ceca.CECA_2P, 0, 4, fused, X_out=oc, Y_out=yc, workspace=ws)
+    assert torch.equal(oc, one)
+
+
+def test_fused_consensus_padded_rows():
+    n, d, ld = 100, 1000, 1024
+    x = synth.consensus_inputs(n, d, seed=9)
+    (X, xb), (Xo, xob), (Yo, yob) = _put(x.to(DEV), ld), _padded(n, d, ld), _padded(n, d, ld)
+    ws = _fused_ws()
+    for variant in (ceca.CECA_2P, ceca.CECA_1P):
+        ceca.ceca_consensus_rounds(X, None, variant, 0, 7, 1, X_out=Xo, Y_out=Yo, workspace=ws)
+        want_x, want_y = oracle.consensus(_np(x), np.zeros((n, d)), variant, 0, 7)
+        tol = STEP_TOL * 7 * float(x.abs().max())
+        assert np.abs(_np(Xo) - want_x).max() <= tol and np.abs(_np(Yo) - want_y).max() <= tol
+        assert torch.isnan(xob[:n * ld].view(n, ld)[:, d:]).all()   # TMA stores clip at column d
+        assert ceca.ceca_read_status(ws) == 0
+
+
+# --------------------------------------------------------------------------------------------
+# logistic gradient
+# --------------------------------------------------------------------------------------------
+
+def _grad_tol(d, want):
+    return 8 * np.sqrt(d) * 2.0 ** -24 * np.abs(want).max() + 1e-7
+
+
+@pytest.mark.parametrize("n,m,d", [(5, 100, 32), (6, 100, 32), (3, 37, 4096), (2, 50, 8192), (2, 33, 1028),
+                                   (4, 16, 2048), (3, 20, 30), (2, 9, 8200), (1, 5, 1), (7, 1, 64)])
+def test_logreg_grad_matches_oracle(n, m, d):
+    a, lab, x_star = synth.logreg_problem(n, m, d, seed=n + m + d, flip=0.1, hetero_std=0.5)
+    gen = torch.Generator().manual_seed(1)
+    x = 0.05 * torch.randn(n, d, generator=gen)
+    y = 0.05 * torch.randn(n, d, generator=gen)
+    A, L, X, Y = a.to(DEV), lab.to(DEV), x.to(DEV), y.to(DEV)
+    ws = torch.empty(ceca.ceca_workspace_bytes(ceca.WS_LOGREG_GRAD, n, m, d) // 4 + 64, dtype=torch.float32, device=DEV)
+    for variant in _variants(n):
+        for k in range(_tau(n)):
+            G = torch.full((n, d), float("nan"), device=DEV)
+            ceca.dsgd_logreg_grad(A, L, X, Y, k, variant, G, ws)
+            want = oracle.logreg_grad(_np(a), _np(lab), _np(x), _np(y), k)
+            assert np.abs(_np(G) - want).max() <= _grad_tol(d, want), (n, m, d, k)
+            G2 = torch.empty_like(G)
+            ceca.dsgd_logreg_grad(A, L, X, Y, k, variant, G2, ws)
+            assert torch.equal(G, G2)  # run-to-run identical
+
+
+@pytest.mark.parametrize("n,variant", [(5, ceca.CECA_2P), (6, ceca.CECA_1P)])
+def test_small_logistic_regression_run(n, variant):
+    """n agents, d = 32, 100 samples each, X0 = Y0 = 0, gamma = 0.05, 60 iterations: gradient kernel
+    + fused step on the GPU against the same loop in the fp64 oracle."""
+    m, d, gamma, iters = 100, 32, 0.05, 60
+    a, lab, _ = synth.logreg_problem(n, m, d, seed=0, flip=0.1)
+    A, L = a.to(DEV), lab.to(DEV)
+    X = torch.zeros(n, d, device=DEV); Y = torch.zeros(n, d, device=DEV); G = torch.empty(n, d, device=DEV)
+    ws = torch.empty(ceca.ceca_workspace_bytes(ceca.WS_LOGREG_GRAD, n, m, d) // 4, dtype=torch.float32, device=DEV)
+    ox = np.zeros((n, d)); oy = np.zeros((n, d))
+    an, ln = _np(a), _np(lab)
+    for k in range(iters):
+        ceca.dsgd_logreg_grad(A, L, X, Y, k, variant, G, ws)
+        ceca.ceca_gossip_sgd_step(X, Y, G, gamma, variant, k)
+        og = oracle.logreg_grad(an, ln, ox, oy, k)
+        ox, oy = oracle.step(ox, oy, og, np.float32(gamma), variant, k)
+        scale = max(np.abs(ox).max(), np.abs(oy).max(), 1e-3)
+        tol = 4e-6 * (k + 1) * scale   # linear growth: each iteration adds a step's and a gradient's rounding
+        assert np.abs(_np(X) - ox).max() <= tol, k
+        assert np.abs(_np(Y) - oy).max() <= tol, k
+    loss0 = oracle.logreg_loss(an, ln, np.zeros((n, d))).mean()
+    loss1 = oracle.logreg_loss(an, ln, np.broadcast_to(_np(X).mean(0), (n, d))).mean()
+    assert loss1 < loss0
+
+
+# --------------------------------------------------------------------------------------------
+# host-memory front end
+# --------------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("pinned", [True, False])
+@pytest.mark.parametrize("n,d,ld,variant", [(6, 1000, 1000, ceca.CECA_1P), (24, 70001, 70004, ceca.CECA_2P),
+                                             (100, 300000, 300000, ceca.CECA_2P)])
+def test_host_step_matches_device_step(pinned, n, d, ld, variant):
+    x, y, g = synth.step_inputs(n, ld, seed=2, x_std=1.0, g_std=1.0, same_xy=False)
+    gamma = 0.1
+    ws = torch.empty(32 << 20, dtype=torch.uint8, device=DEV)
+    for k in range(_tau(n)):
+        hx, hy, hg = x.clone(), y.clone(), g.clone()
+        if pinned:
+            hx, hy, hg = hx.pin_memory(), hy.pin_memory(), hg.pin_memory()
+        ceca.ceca_gossip_sgd_step_host(hx[:, :d], hy[:, :d], hg[:, :d], gamma, variant, k, ws)
+        X, Y, G = x[:, :d].to(DEV).contiguous(), y[:, :d].to(DEV).contiguous(), g[:, :d].to(DEV).contiguous()
+        ceca.ceca_gossip_sgd_step(X, Y, G, gamma, variant, k)
+        assert torch.equal(hx[:, :d], X.cpu()) and torch.equal(hy[:, :d], Y.cpu())
+        assert torch.equal(hx[:, d:], x[:, d:]) and torch.equal(hg, g)   # padding and G untouched
+
+
+# --------------------------------------------------------------------------------------------
+# full-size workloads, checked on column windows (columns never interact in the update)
+# --------------------------------------------------------------------------------------------
+
+def _windows(d, width, count, seed):
+    rng = np.random.default_rng(seed)
+    starts = [0, max(d - width, 0)] + [int(s) for s in rng.integers(0, max(d - width, 1), size=count)]
+    return [(s, min(s + width, d)) for s in starts]
+
+
+def _need_free(bytes_needed):
+    free, _ = torch.cuda.mem_get_info()
+    if free < bytes_needed:
+        pytest.skip("needs %.1f GB of free device memory" % (bytes_needed / 1e9))
+
+
+@pytest.mark.parametrize("n,d,variant,iters", [(24, 11_689_512, ceca.CECA_1P, 5), (100, 25_557_032, ceca.CECA_2P, 7)])
+def test_full_size_step_on_column_windows(n, d, variant, iters):
+    """Flat CNN-sized parameter vectors (ResNet-18 / ResNet-50 sized), in place, the launch shape the
+    benchmark times; windows include the first and the last (ragged) columns."""
+    _need_free(int(3.3 * n * d * 4))
+    X, Y, G = synth.step_inputs(n, d, seed=4, x_std=0.01, g_std=0.01, device=DEV)
+    gamma = 0.1
+    wins = _windows(d, 4099, 4, seed=n)
+    ref = [(_np(X[:, lo:hi]).astype(np.float64), _np(Y[:, lo:hi]).astype(np.float64)) for lo, hi in wins]
+    for k in range(iters):
+        synth.gradient_inputs(n, d, k, g_std=0.01, device=DEV, out=G)
+        gw = [_np(G[:, lo:hi]) for lo, hi in wins]
+        before = [( _np(X[:, lo:hi]), _np(Y[:, lo:hi])) for lo, hi in wins]
+        ceca.ceca_gossip_sgd_step(X, Y, G, gamma, variant, k)
+        for w, (lo, hi) in enumerate(wins):
+            want_x, want_y = oracle.step(before[w][0], before[w][1], gw[w], np.float32(gamma), variant, k)
+            tol = STEP_TOL * max(np.abs(before[w][0]).max(), np.abs(before[w][1]).max())
+            assert np.abs(_np(X[:, lo:hi]) - want_x).max() <= tol, (k, lo)
+            assert np.abs(_np(Y[:, lo:hi]) - want_y).max() <= tol, (k, lo)
+            # and the whole trajectory against an fp64 run from the same start
+            ref[w] = oracle.step(ref[w][0], ref[w][1], gw[w], np.float32(gamma), variant, k)
+            assert np.abs(_np(X[:, lo:hi]) - ref[w][0]).max() <= tol * (k + 1)
+
+
+@pytest.mark.parametrize("fused", [0, 1])
+def test_full_size_consensus_on_column_windows(fused):
+    """n = 97 (prime), d = 2^20, rows offset by the agent index, tau = 7 rounds, 2-port."""
+    n, d, tau = 97, 1 << 20, 7
+    x = synth.consensus_inputs(n, d, seed=1, device=DEV)
+    Xo, Yo = torch.empty_like(x), torch.empty_like(x)
+    ws = _fused_ws()
+    ceca.ceca_consensus_rounds(x, None, ceca.CECA_2P, 0, tau, fused, X_out=Xo, Y_out=Yo, workspace=ws)
+    assert ceca.ceca_read_status(ws) == 0
+    xd = Xo.double()
+    mean = x.double().mean(0)
+    assert float((xd - mean).norm() / xd.norm()) <= 1e-5
+    for lo, hi in _windows(d, 2048, 4, seed=97):
+        want_x, want_y = oracle.consensus(_np(x[:, lo:hi]), np.zeros((n, hi - lo)), ceca.CECA_2P, 0, tau)
+        tol = STEP_TOL * tau * float(x.abs().max())
+        assert np.abs(_np(Xo[:, lo:hi]) - want_x).max() <= tol
+        assert np.abs(_np(Yo[:, lo:hi]) - want_y).max() <= tol
+
+
+def test_heterogeneous_logreg_full_size_first_iterations():
+    """n = 63, 2000 samples, d = 4096, per-agent feature shifts: gradient + fused step, 2-port, checked
+    against the oracle for the first iterations."""
+    n, m, d, gamma = 63, 2000, 4096, 0.01
+    _need_free(int(1.3 * n * m * d * 4))
+    A, L, _ = synth.logreg_problem(n, m, d, seed=3, flip=0.05, hetero_std=0.5, device=DEV)
+    X = torch.zeros(n, d, device=DEV); Y = torch.zeros(n, d, device=DEV); G = torch.empty(n, d, device=DEV)
+    ws = torch.empty(ceca.ceca_workspace_bytes(ceca.WS_LOGREG_GRAD, n, m, d) // 4, dtype=torch.float32, device=DEV)
+    agents = [0, 31, 62]
+    an = {i: _np(A[i:i + 1]) for i in agents}
+    ln = {i: _np(L[i:i + 1]) for i in agents}
+    for k in range(4):
+        ceca.dsgd_logreg_grad(A, L, X, Y, k, ceca.CECA_2P, G, ws)
+        z = Y if oracle.round_info(n, k).payload else X
+        for i in agents:   # the gradient of agent i depends on its own data and model only
+            zi = _np(z[i:i + 1])
+            want = oracle.logreg_grad(an[i], ln[i], zi, zi, 0)
+            assert np.abs(_np(G[i:i + 1]) - want).max() <= _grad_tol(d, want), (k, i)
+        bx, by, bg = _np(X), _np(Y), _np(G)
+        ceca.ceca_gossip_sgd_step(X, Y, G, gamma, ceca.CECA_2P, k)
+        want_x, want_y = oracle.step(bx, by, bg, np.float32(gamma), ceca.CECA_2P, k)
+        tol = STEP_TOL * max(np.abs(bx).max(), np.abs(by).max(), gamma * np.abs(bg).max())
+        assert np.abs(_np(X) - want_x).max() <= tol and np.abs(_np(Y) - want_y).max() <= tol

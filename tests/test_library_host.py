@@ -1,0 +1,111 @@
+"""Host-side checks of the CUDA library that need no GPU: exported symbols, the schedule
+(bit-exact against the oracle), error codes and workspace sizes."""
+import ctypes
+import os
+import re
+
+import numpy as np
+import pytest
+
+import oracle
+import paper_2306_00256_b200 as ceca
+from paper_2306_00256_b200 import binding
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _declared_functions():
+    text = open(os.path.join(ROOT, "include", "ceca.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b((?:ceca|dsgd)_[a-z_]+)\s*\(", text)))
+
+
+def test_library_loads_and_exports_every_declared_symbol():
+    lib = ceca.library()
+    declared = _declared_functions()
+    assert {"ceca_schedule", "ceca_gossip_sgd_step", "ceca_consensus_rounds", "dsgd_logreg_grad"} <= set(declared)
+    for name in declared:
+        assert hasattr(lib, name), name
+    assert sorted(binding.EXPORTS) == declared
+
+
+def test_round_struct_layout_matches_header():
+    assert ctypes.sizeof(ceca.Round) == 10 * 4 + 2 * 8
+    assert ceca.Round.a.offset == 40
+
+
+@pytest.mark.parametrize("variant", [ceca.CECA_1P, ceca.CECA_2P])
+def test_schedule_bit_exact_against_oracle(variant):
+    sizes = list(range(1, 600)) + [1023, 1024, 1025, 1026, 2047, 2048, 2049, 4095, 4096, 65536, 99991, 100000]
+    for n in sizes:
+        if variant == ceca.CECA_1P and n % 2 and n > 1:
+            continue
+        tau = oracle.round_info(n, 0).tau
+        for r in range(max(tau, 1)):
+            rd, recv, send = ceca.ceca_schedule(n, variant, r)
+            want = oracle.round_info(n, r)
+            for f, _ in ceca.Round._fields_:
+                assert getattr(rd, f) == getattr(want, f), (n, r, f)
+            assert np.float64(rd.a).tobytes() == np.float64(want.a).tobytes()
+            assert np.float64(rd.b).tobytes() == np.float64(want.b).tobytes()
+            want_recv, want_send = oracle.peers(n, variant, r)
+            assert np.array_equal(recv, want_recv) and np.array_equal(send, want_send), (n, r)
+
+
+def test_schedule_large_iteration_counter():
+    for n in (2, 6, 97, 100):
+        for k in (2**31 - 1, 2**31, 2**31 + 5, 2**40 + 3, 2**62 + 11):
+            for variant in (ceca.CECA_1P, ceca.CECA_2P):
+                if variant == ceca.CECA_1P and n % 2:
+                    continue
+                rd, recv, send = ceca.ceca_schedule(n, variant, k)
+                want = oracle.round_info(n, k)
+                assert (rd.r, rd.delta, rd.n_r) == (want.r, want.delta, want.n_r)
+                assert np.array_equal(recv, oracle.peers(n, variant, k)[0])
+
+
+def test_schedule_errors():
+    for n, variant, k, status in [(0, 2, 0, 1), (-3, 2, 0, 1), (6, 2, -1, 1), (6, 3, 0, 1), (6, 0, 0, 1),
+                                  (5, 1, 0, 2), (97, 1, 3, 2)]:
+        with pytest.raises(ceca.CecaError) as err:
+            ceca.ceca_schedule(n, variant, k)
+        assert err.value.status == status
+    rd, recv, send = ceca.ceca_schedule(1, ceca.CECA_1P, 7)   # a single agent is fine in both variants
+    assert (rd.tau, rd.a, rd.b) == (0, 1.0, 1.0) and recv[0] == 0 and send[0] == 0
+    rd, recv, send = ceca.ceca_schedule(6, ceca.CECA_2P, 1, peers=False)
+    assert recv is None and rd.payload == 1
+
+
+def test_device_entry_points_reject_bad_arguments_before_touching_the_gpu():
+    lib = ceca.library()
+    fake = ctypes.c_void_p(256)  # never dereferenced: every call below fails validation first
+    step = lib.ceca_gossip_sgd_step
+    assert step(None, fake, fake, fake, fake, 4, 8, 8, 0.1, 2, 0, None) == 1
+    assert step(fake, fake, fake, fake, fake, 0, 8, 8, 0.1, 2, 0, None) == 1
+    assert step(fake, fake, fake, fake, fake, 4, 8, 7, 0.1, 2, 0, None) == 1      # ld < d
+    assert step(fake, fake, fake, fake, fake, 5, 8, 8, 0.1, 1, 0, None) == 2      # odd n, 1-port
+    assert step(fake, None, fake, fake, ctypes.c_void_p(512), 4, 8, 8, 0.1, 2, 1, None) == 1  # round 1 needs Y
+    assert step(fake, fake, None, fake, fake, 4, 8, 8, 0.1, 2, 1, None) == 4      # X_out == Y_out
+    cons = lib.ceca_consensus_rounds
+    assert cons(fake, fake, fake, fake, 4, 8, 8, 2, 0, -1, 0, None, 0, None) == 1
+    assert cons(fake, None, ctypes.c_void_p(512), None, 4, 8, 8, 2, 0, 2, 0, None, 0, None) == 5  # no Y_out, no workspace
+    assert cons(fake, None, ctypes.c_void_p(512), None, 300, 8, 8, 2, 0, 2, 1, fake, 256, None) == 4  # n > 256 fused
+    assert cons(fake, None, ctypes.c_void_p(516), None, 4, 8, 8, 2, 0, 2, 1, fake, 256, None) == 3  # misaligned
+    assert cons(fake, None, ctypes.c_void_p(512), None, 4, 8, 6, 2, 0, 2, 1, fake, 256, None) == 1  # ld < d
+    assert cons(fake, None, ctypes.c_void_p(512), None, 4, 6, 6, 2, 0, 2, 1, fake, 256, None) == 3  # ld*4 % 16
+    assert cons(fake, None, ctypes.c_void_p(512), None, 4, 8, 8, 2, 1, 2, 1, fake, 256, None) == 1  # starts at r=1, no Y
+    grad = lib.dsgd_logreg_grad
+    assert grad(fake, fake, fake, fake, 0, fake, 4, 0, 8, 8, 2, fake, 1 << 20, None) == 1
+    assert grad(fake, fake, fake, fake, 0, fake, 4, 5, 8, 8, 2, None, 0, None) == 5
+    assert grad(fake, fake, fake, None, 1, fake, 6, 5, 8, 8, 2, fake, 1 << 20, None) == 1  # n=6, k=1 evaluates at Y
+    host = lib.ceca_gossip_sgd_step_host
+    assert host(fake, fake, fake, 4, 8, 8, 0.1, 2, 0, None, 0) == 5
+    assert host(fake, fake, fake, 5, 8, 8, 0.1, 1, 0, fake, 1 << 20) == 2
+
+
+def test_workspace_sizes():
+    assert ceca.ceca_workspace_bytes(ceca.WS_CONSENSUS_FUSED, 97, 0, 1 << 20) >= 4
+    assert ceca.ceca_workspace_bytes(ceca.WS_CONSENSUS_UNFUSED, 97, 0, 1024) == 97 * 1024 * 4
+    assert ceca.ceca_workspace_bytes(ceca.WS_LOGREG_GRAD, 63, 2000, 4096) >= 63 * 2000 * 4
+    assert ceca.ceca_workspace_bytes(ceca.WS_STEP_HOST, 100, 0, 1 << 20) >= 3 * 3 * 100 * 4 * 4
+    assert ceca.ceca_status_string(0) == "ok" and "even" in ceca.ceca_status_string(2)
