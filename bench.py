@@ -48,7 +48,12 @@ WORKLOADS = {
 FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
 # capture summarised under profiles/ (None until captured, or once the kernel has changed since).
-NCU_TRAFFIC_BYTES_PER_LAUNCH = {}
+NCU_TRAFFIC_BYTES_PER_LAUNCH = {
+    # 19.75 B per agent-parameter measured on step_small (2.5167 GB read + 1.6243 GB written for
+    # 100 x 2,097,152 units); traffic is proportional to the units, scaled here to n*d of each workload
+    "step_small": 4.141e9,
+    "resnet50_step": 19.746 * 100 * 25_557_032,
+}
 
 
 def measured_peak():
