@@ -222,7 +222,9 @@ def bench_step(args, wl, device, dist):
                 "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH.get(args.workload),
                 "kernel": "step_walk_kernel<float4, gradient, reads Y>", "peak_source": "of " + which,
                 "avg_launch_ms": avg_ms, "launches_timed": len(dominant),
-                "frac_of_nominal_8TBs": achieved / 8000.0}
+                "frac_of_nominal_8TBs": achieved / 8000.0,
+                "ms_by_round": [round(statistics.mean(per_launch[s] for s in range(args.steps) if (k_first + s) % tau == r), 4)
+                                if any((k_first + s) % tau == r for s in range(args.steps)) else None for r in range(tau)]}
     del X, Y, G
     torch.cuda.empty_cache()
     return total_ms, launches, roof, clocks, {"tau": tau, "in_place": True, "l2": "inputs (3 x n x d fp32) far larger than L2"}

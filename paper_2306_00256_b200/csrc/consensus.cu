@@ -6,9 +6,11 @@
 //   thread keeps a few rows of one column for the whole run), and runs all rounds on chip: per
 //   round every thread publishes the payload (I or J) of its rows in a shared exchange buffer,
 //   the CTA synchronises, and every thread picks up the value of the row it receives from.  Only
-//   4 bytes per element per round go through shared memory in each direction.  The finished
-//   tiles go back with one TMA tensor store each.  HBM sees X once in and X (and Y) once out,
-//   instead of once per round.
+//   4 bytes per element per round go through shared memory in each direction.  A thread owns four
+//   adjacent columns (128-bit shared-memory accesses, packed two-wide fp32 FMAs), which keeps the
+//   instruction count per element low enough for the kernel to be bound by memory and not by
+//   issue slots.  The finished tiles go back with one TMA tensor store each.  HBM sees X once in
+//   and X (and Y) once out, instead of once per round.
 #include <cuda.h>
 #include <cuda_runtime.h>
 
@@ -28,8 +30,9 @@ ceca_status_t check_matrix_args(const void *X, const void *X_out, int32_t n, int
 constexpr int kMaxFusedRounds = 64;
 constexpr int kMaxFusedRows = 256;   // one TMA box holds at most 256 rows
 constexpr int kTileCols = 32;        // W: columns per CTA tile (128-byte row segments)
-constexpr int kRowGroups = 8;        // Q: a column's rows are dealt round-robin to Q threads
-constexpr int kFusedThreads = kTileCols * kRowGroups;
+constexpr int kFusedThreads = 256;
+constexpr int kColGroups = kTileCols / 4;                 // a thread owns 4 adjacent columns
+constexpr int kRowGroups = kFusedThreads / kColGroups;    // Q: rows are dealt round-robin to Q threads
 constexpr uint32_t kWaitPolls = 1u << 22;  // bounded mbarrier wait (each poll sleeps ~100 ns)
 
 struct FusedRound {
@@ -87,6 +90,14 @@ __device__ __forceinline__ void tma_store_2d(const CUtensorMap *map, int32_t x, 
                : "memory");
 }
 
+__device__ __forceinline__ float4 mix4(float w_own, float4 own, float w_recv, float4 recv) {
+  // w_own * own + w_recv * recv on four lanes with two-wide packed fp32 instructions
+  const float2 wo = make_float2(w_own, w_own), wr = make_float2(w_recv, w_recv);
+  const float2 lo = __ffma2_rn(wo, make_float2(own.x, own.y), __fmul2_rn(wr, make_float2(recv.x, recv.y)));
+  const float2 hi = __ffma2_rn(wo, make_float2(own.z, own.w), __fmul2_rn(wr, make_float2(recv.z, recv.w)));
+  return make_float4(lo.x, lo.y, hi.x, hi.y);
+}
+
 // R = rows per thread (compile time), so n <= R * kRowGroups.
 template <int R>
 __global__ void __launch_bounds__(kFusedThreads)
@@ -99,8 +110,8 @@ consensus_fused_kernel(const __grid_constant__ CUtensorMap map_x_in, const __gri
   float *tile_b = tile_a + (size_t)n * kTileCols;                 // [n][W]  Y tile, then exchange buffer 1
   __shared__ __align__(8) uint64_t bar;
 
-  const int c = threadIdx.x % kTileCols;
-  const int q = threadIdx.x / kTileCols;
+  const int c = (threadIdx.x % kColGroups) * 4;  // first of this thread's four columns
+  const int q = threadIdx.x / kColGroups;
   const int32_t col0 = (int32_t)blockIdx.x * kTileCols;  // multiple of 32 floats: 16-byte aligned
 
   if (threadIdx.x == 0) {
@@ -123,22 +134,31 @@ consensus_fused_kernel(const __grid_constant__ CUtensorMap map_x_in, const __gri
     return;
   }
 
-  float I[R], J[R];
+  float4 I[R], J[R];
 #pragma unroll
   for (int t = 0; t < R; ++t) {
     const int i = q + t * kRowGroups;
-    I[t] = i < n ? tile_a[i * kTileCols + c] : 0.f;
-    J[t] = (i < n && p.has_y_in) ? tile_b[i * kTileCols + c] : 0.f;
+    const float4 zero = make_float4(0.f, 0.f, 0.f, 0.f);
+    I[t] = i < n ? *reinterpret_cast<const float4 *>(tile_a + i * kTileCols + c) : zero;
+    J[t] = (i < n && p.has_y_in) ? *reinterpret_cast<const float4 *>(tile_b + i * kTileCols + c) : zero;
   }
   __syncthreads();  // both tiles are now free to serve as exchange buffers
 
   for (int rnd = 0; rnd < p.rounds; ++rnd) {
     const FusedRound rd = p.rd[rnd];
     float *buf = (rnd & 1) ? tile_b : tile_a;
+    if (rd.payload) {
 #pragma unroll
-    for (int t = 0; t < R; ++t) {
-      const int i = q + t * kRowGroups;
-      if (i < n) buf[i * kTileCols + c] = rd.payload ? J[t] : I[t];
+      for (int t = 0; t < R; ++t) {
+        const int i = q + t * kRowGroups;
+        if (i < n) *reinterpret_cast<float4 *>(buf + i * kTileCols + c) = J[t];
+      }
+    } else {
+#pragma unroll
+      for (int t = 0; t < R; ++t) {
+        const int i = q + t * kRowGroups;
+        if (i < n) *reinterpret_cast<float4 *>(buf + i * kTileCols + c) = I[t];
+      }
     }
     __syncthreads();
 #pragma unroll
@@ -148,9 +168,9 @@ consensus_fused_kernel(const __grid_constant__ CUtensorMap map_x_in, const __gri
         int src;
         if (p.one_port && !(i & 1)) { src = i + rd.hop; if (src >= n) src -= n; }
         else                        { src = i - rd.hop; if (src < 0) src += n; }
-        const float recv = buf[src * kTileCols + c];
-        I[t] = fmaf(rd.a, I[t], rd.one_minus_a * recv);
-        J[t] = fmaf(rd.b, J[t], rd.one_minus_b * recv);
+        const float4 recv = *reinterpret_cast<const float4 *>(buf + src * kTileCols + c);
+        I[t] = mix4(rd.a, I[t], rd.one_minus_a, recv);
+        J[t] = mix4(rd.b, J[t], rd.one_minus_b, recv);
       }
     }
     // no second barrier: the next round writes the other buffer, and a thread can only start
@@ -162,8 +182,8 @@ consensus_fused_kernel(const __grid_constant__ CUtensorMap map_x_in, const __gri
   for (int t = 0; t < R; ++t) {
     const int i = q + t * kRowGroups;
     if (i < n) {
-      tile_a[i * kTileCols + c] = I[t];
-      if (p.has_y_out) tile_b[i * kTileCols + c] = J[t];
+      *reinterpret_cast<float4 *>(tile_a + i * kTileCols + c) = I[t];
+      if (p.has_y_out) *reinterpret_cast<float4 *>(tile_b + i * kTileCols + c) = J[t];
     }
   }
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic writes -> visible to TMA
@@ -255,14 +275,14 @@ static ceca_status_t consensus_fused(const float *X, const float *Y, float *Xo, 
   if (!make_map(&myi, args.has_y_in ? Y : X, n, d, ld)) return CECA_ERR_CUDA;
   if (!make_map(&myo, Yo ? Yo : Xo, n, d, ld)) return CECA_ERR_CUDA;
 
-  const int rows_per_thread = (n + kRowGroups - 1) / kRowGroups;
+  const int rows_per_thread = (n + kRowGroups - 1) / kRowGroups;  // n <= 256 -> at most 8
   cudaError_t e;
-  if (rows_per_thread <= 4)       e = launch_fused<4>(mxi, myi, mxo, myo, args, d, stream);
-  else if (rows_per_thread <= 8)  e = launch_fused<8>(mxi, myi, mxo, myo, args, d, stream);
-  else if (rows_per_thread <= 13) e = launch_fused<13>(mxi, myi, mxo, myo, args, d, stream);
-  else if (rows_per_thread <= 16) e = launch_fused<16>(mxi, myi, mxo, myo, args, d, stream);
-  else if (rows_per_thread <= 24) e = launch_fused<24>(mxi, myi, mxo, myo, args, d, stream);
-  else                            e = launch_fused<32>(mxi, myi, mxo, myo, args, d, stream);
+  if (rows_per_thread <= 1)      e = launch_fused<1>(mxi, myi, mxo, myo, args, d, stream);
+  else if (rows_per_thread <= 2) e = launch_fused<2>(mxi, myi, mxo, myo, args, d, stream);
+  else if (rows_per_thread <= 3) e = launch_fused<3>(mxi, myi, mxo, myo, args, d, stream);
+  else if (rows_per_thread <= 4) e = launch_fused<4>(mxi, myi, mxo, myo, args, d, stream);
+  else if (rows_per_thread <= 6) e = launch_fused<6>(mxi, myi, mxo, myo, args, d, stream);
+  else                           e = launch_fused<8>(mxi, myi, mxo, myo, args, d, stream);
   return e == cudaSuccess ? CECA_OK : CECA_ERR_CUDA;
 }
 

@@ -48,7 +48,6 @@ template <typename V> __device__ __forceinline__ void vstore(float *p, V v) {
 }
 
 constexpr int kThreads = 256;
-constexpr int kRowsInFlight = 4;  // rows whose loads are issued before any of them is consumed
 
 // One row's own terms: own_x = x - gamma e, own_y = y - gamma e, and the message u (one of them).
 template <typename V, bool HAS_G, bool USE_Y>
@@ -66,8 +65,11 @@ struct RowRegs {
   }
 };
 
-template <typename V, bool HAS_G, bool USE_Y>
-__global__ void __launch_bounds__(kThreads) step_walk_kernel(const StepArgs p) {
+// RIF = rows whose loads are issued before any of them is consumed (memory-level parallelism per
+// thread); MINB = CTAs per SM the register allocation must allow (parallelism across threads).
+// Long cycles want a deep RIF, cycles of two rows have only two rows to load and want occupancy.
+template <typename V, bool HAS_G, bool USE_Y, int RIF, int MINB>
+__global__ void __launch_bounds__(kThreads, MINB) step_walk_kernel(const StepArgs p) {
   constexpr int VW = sizeof(V) / sizeof(float);
   const int64_t colv = (int64_t)blockIdx.x * kThreads + threadIdx.x;
   if (colv >= p.ncolv) return;
@@ -83,11 +85,11 @@ __global__ void __launch_bounds__(kThreads) step_walk_kernel(const StepArgs p) {
     V first_own_x, first_own_y, u_prev;
     bool first_done = false;
     int32_t row = first_row;
-    for (int32_t t = 1; t < p.cycle_len; t += kRowsInFlight) {
-      Row batch[kRowsInFlight];
-      int64_t offs[kRowsInFlight];
+    for (int32_t t = 1; t < p.cycle_len; t += RIF) {
+      Row batch[RIF];
+      int64_t offs[RIF];
 #pragma unroll
-      for (int j = 0; j < kRowsInFlight; ++j) {
+      for (int j = 0; j < RIF; ++j) {
         if (t + j < p.cycle_len) {
           row += p.hop;
           if (row >= p.n) row -= p.n;
@@ -100,7 +102,7 @@ __global__ void __launch_bounds__(kThreads) step_walk_kernel(const StepArgs p) {
         first_done = true;
       }
 #pragma unroll
-      for (int j = 0; j < kRowsInFlight; ++j) {
+      for (int j = 0; j < RIF; ++j) {
         if (t + j < p.cycle_len) {
           V own_x, own_y, u;
           batch[j].own_terms(p, own_x, own_y, u);
@@ -117,20 +119,32 @@ __global__ void __launch_bounds__(kThreads) step_walk_kernel(const StepArgs p) {
   }
 }
 
-template <typename V>
-static cudaError_t launch_walk(const StepArgs &args, bool has_g, bool use_y, cudaStream_t stream) {
-  if (args.ncolv <= 0) return cudaSuccess;
+template <typename V, int RIF, int MINB>
+static cudaError_t launch_walk_shape(const StepArgs &args, bool has_g, bool use_y, cudaStream_t stream) {
   const int64_t blocks_x = (args.ncolv + kThreads - 1) / kThreads;
   if (blocks_x > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
   dim3 grid((unsigned)blocks_x, (unsigned)(args.n_cycles < 65535 ? args.n_cycles : 65535));
   if (has_g) {
-    if (use_y) step_walk_kernel<V, true, true><<<grid, kThreads, 0, stream>>>(args);
-    else       step_walk_kernel<V, true, false><<<grid, kThreads, 0, stream>>>(args);
+    if (use_y) step_walk_kernel<V, true, true, RIF, MINB><<<grid, kThreads, 0, stream>>>(args);
+    else       step_walk_kernel<V, true, false, RIF, MINB><<<grid, kThreads, 0, stream>>>(args);
   } else {
-    if (use_y) step_walk_kernel<V, false, true><<<grid, kThreads, 0, stream>>>(args);
-    else       step_walk_kernel<V, false, false><<<grid, kThreads, 0, stream>>>(args);
+    if (use_y) step_walk_kernel<V, false, true, RIF, MINB><<<grid, kThreads, 0, stream>>>(args);
+    else       step_walk_kernel<V, false, false, RIF, MINB><<<grid, kThreads, 0, stream>>>(args);
   }
   return cudaGetLastError();
+}
+
+// Launch shapes, chosen from a sweep on a B200 at n = 100, d = 25.6M and n = 24, d = 11.7M:
+// cycles of two rows (every CECA-1P round, and the 2-port shift n/2) have nothing to pipeline and
+// run fastest with many resident CTAs; long walks want four rows of loads in flight per thread.
+template <typename V>
+static cudaError_t launch_walk(const StepArgs &args, bool has_g, bool use_y, cudaStream_t stream) {
+  if (args.ncolv <= 0) return cudaSuccess;
+  if (args.cycle_len <= 2)
+    return use_y ? launch_walk_shape<V, 1, 4>(args, has_g, use_y, stream)
+                 : launch_walk_shape<V, 1, 6>(args, has_g, use_y, stream);
+  if (args.cycle_len <= 4) return launch_walk_shape<V, 2, 4>(args, has_g, use_y, stream);
+  return launch_walk_shape<V, 4, 2>(args, has_g, use_y, stream);
 }
 
 static inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
