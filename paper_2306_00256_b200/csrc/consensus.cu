@@ -3,14 +3,14 @@
 // fused = 0: one pass of the step kernel (gamma = 0, no G) per round.
 // fused = 1: one launch.  Each CTA brings an n x W column tile of X (and of Y when the first
 //   round needs it) into shared memory with one TMA tensor load, moves it into registers (a
-//   thread keeps a few rows of one column for the whole run), and runs all rounds on chip: per
+//   thread keeps a few rows of eight columns for the whole run), and runs all rounds on chip: per
 //   round every thread publishes the payload (I or J) of its rows in a shared exchange buffer,
 //   the CTA synchronises, and every thread picks up the value of the row it receives from.  Only
-//   4 bytes per element per round go through shared memory in each direction.  A thread owns four
-//   adjacent columns (128-bit shared-memory accesses, packed two-wide fp32 FMAs), which keeps the
-//   instruction count per element low enough for the kernel to be bound by memory and not by
-//   issue slots.  The finished tiles go back with one TMA tensor store each.  HBM sees X once in
-//   and X (and Y) once out, instead of once per round.
+//   4 bytes per element per round go through shared memory in each direction (128-bit accesses,
+//   packed two-wide fp32 FMAs; eight columns per thread keep the index arithmetic per element
+//   small).  The finished tiles go back with one TMA tensor store each.  HBM sees X once in and
+//   X (and Y) once out, instead of once per round.  Several CTAs per SM overlap each other's
+//   load, compute and store phases.
 #include <cuda.h>
 #include <cuda_runtime.h>
 
@@ -31,8 +31,8 @@ constexpr int kMaxFusedRounds = 64;
 constexpr int kMaxFusedRows = 256;   // one TMA box holds at most 256 rows
 constexpr int kTileCols = 32;        // W: columns per CTA tile (128-byte row segments)
 constexpr int kFusedThreads = 256;
-constexpr int kColGroups = kTileCols / 4;                 // a thread owns 4 adjacent columns
-constexpr int kRowGroups = kFusedThreads / kColGroups;    // Q: rows are dealt round-robin to Q threads
+constexpr int kColGroups = 4;                             // a thread owns 2 x 4 columns: groups cg and cg + 4
+constexpr int kRowGroups = kFusedThreads / kColGroups;    // Q = 64: rows are dealt round-robin to Q threads
 constexpr uint32_t kWaitPolls = 1u << 22;  // bounded mbarrier wait (each poll sleeps ~100 ns)
 
 struct FusedRound {
@@ -99,6 +99,12 @@ __device__ __forceinline__ float4 mix4(float w_own, float4 own, float w_recv, fl
 }
 
 // R = rows per thread (compile time), so n <= R * kRowGroups.
+//
+// Thread layout: cg = tid % 4, q = tid / 4.  A thread owns rows q, q + 64, ... and, in each, the two
+// float4 column groups cg and cg + 4 (columns 4 cg .. 4 cg + 3 and 16 + 4 cg .. 16 + 4 cg + 3).
+// It touches them in the order (cg, cg + 4) when q is even and (cg + 4, cg) when q is odd, so the
+// eight threads that share a 128-bit shared-memory transaction (two adjacent row groups) cover
+// all 32 banks: rows are 128 bytes apart and would otherwise collide.
 template <int R>
 __global__ void __launch_bounds__(kFusedThreads)
 consensus_fused_kernel(const __grid_constant__ CUtensorMap map_x_in, const __grid_constant__ CUtensorMap map_y_in,
@@ -106,12 +112,14 @@ consensus_fused_kernel(const __grid_constant__ CUtensorMap map_x_in, const __gri
                        const __grid_constant__ CUtensorMap map_y_out, const __grid_constant__ FusedArgs p) {
   extern __shared__ __align__(128) unsigned char smem_raw[];
   const int n = p.n;
-  float *tile_a = reinterpret_cast<float *>(smem_raw);            // [n][W]  X tile, then exchange buffer 0
-  float *tile_b = tile_a + (size_t)n * kTileCols;                 // [n][W]  Y tile, then exchange buffer 1
+  float *tile_a = reinterpret_cast<float *>(smem_raw);            // [n][W]  X tile, then exchange buffer
+  float *tile_b = tile_a + (size_t)n * kTileCols;                 // [n][W]  Y tile, then exchange buffer
   __shared__ __align__(8) uint64_t bar;
 
-  const int c = (threadIdx.x % kColGroups) * 4;  // first of this thread's four columns
+  const int cg = threadIdx.x % kColGroups;
   const int q = threadIdx.x / kColGroups;
+  const int c0 = 4 * (cg + 4 * (q & 1));        // columns of the float4 touched first
+  const int c1 = 4 * (cg + 4 * ((q & 1) ^ 1));  // ... and second
   const int32_t col0 = (int32_t)blockIdx.x * kTileCols;  // multiple of 32 floats: 16-byte aligned
 
   if (threadIdx.x == 0) {
@@ -134,33 +142,52 @@ consensus_fused_kernel(const __grid_constant__ CUtensorMap map_x_in, const __gri
     return;
   }
 
-  float4 I[R], J[R];
+  float4 I0[R], I1[R], J0[R], J1[R];
 #pragma unroll
   for (int t = 0; t < R; ++t) {
     const int i = q + t * kRowGroups;
     const float4 zero = make_float4(0.f, 0.f, 0.f, 0.f);
-    I[t] = i < n ? *reinterpret_cast<const float4 *>(tile_a + i * kTileCols + c) : zero;
-    J[t] = (i < n && p.has_y_in) ? *reinterpret_cast<const float4 *>(tile_b + i * kTileCols + c) : zero;
+    I0[t] = I1[t] = J0[t] = J1[t] = zero;
+    if (i < n) {
+      I0[t] = *reinterpret_cast<const float4 *>(tile_a + i * kTileCols + c0);
+      I1[t] = *reinterpret_cast<const float4 *>(tile_a + i * kTileCols + c1);
+      if (p.has_y_in) {
+        J0[t] = *reinterpret_cast<const float4 *>(tile_b + i * kTileCols + c0);
+        J1[t] = *reinterpret_cast<const float4 *>(tile_b + i * kTileCols + c1);
+      }
+    }
   }
-  __syncthreads();  // both tiles are now free to serve as exchange buffers
+  // The landed tiles double as the first round's exchange buffer: if that round sends I it reads
+  // tile_a as it is, if it sends J it reads tile_b (present whenever J carries data).  Later rounds
+  // alternate between the two tiles, starting with the one the first round does not read.
+  const int first_buf = (p.rounds > 0 && p.rd[0].payload && p.has_y_in) ? 1 : 0;
+  const bool first_free = p.rounds > 0 && (!p.rd[0].payload || p.has_y_in);
 
   for (int rnd = 0; rnd < p.rounds; ++rnd) {
     const FusedRound rd = p.rd[rnd];
-    float *buf = (rnd & 1) ? tile_b : tile_a;
-    if (rd.payload) {
+    float *buf = ((rnd + first_buf) & 1) ? tile_b : tile_a;
+    if (rnd == 0 && first_free) {
+      // nothing to publish: every thread has passed the landing barrier, the tile is complete
+    } else if (rd.payload) {
 #pragma unroll
       for (int t = 0; t < R; ++t) {
         const int i = q + t * kRowGroups;
-        if (i < n) *reinterpret_cast<float4 *>(buf + i * kTileCols + c) = J[t];
+        if (i < n) {
+          *reinterpret_cast<float4 *>(buf + i * kTileCols + c0) = J0[t];
+          *reinterpret_cast<float4 *>(buf + i * kTileCols + c1) = J1[t];
+        }
       }
     } else {
 #pragma unroll
       for (int t = 0; t < R; ++t) {
         const int i = q + t * kRowGroups;
-        if (i < n) *reinterpret_cast<float4 *>(buf + i * kTileCols + c) = I[t];
+        if (i < n) {
+          *reinterpret_cast<float4 *>(buf + i * kTileCols + c0) = I0[t];
+          *reinterpret_cast<float4 *>(buf + i * kTileCols + c1) = I1[t];
+        }
       }
     }
-    __syncthreads();
+    __syncthreads();  // payloads visible; in round 0 also: everybody has taken its own rows out
 #pragma unroll
     for (int t = 0; t < R; ++t) {
       const int i = q + t * kRowGroups;
@@ -168,22 +195,29 @@ consensus_fused_kernel(const __grid_constant__ CUtensorMap map_x_in, const __gri
         int src;
         if (p.one_port && !(i & 1)) { src = i + rd.hop; if (src >= n) src -= n; }
         else                        { src = i - rd.hop; if (src < 0) src += n; }
-        const float4 recv = *reinterpret_cast<const float4 *>(buf + src * kTileCols + c);
-        I[t] = mix4(rd.a, I[t], rd.one_minus_a, recv);
-        J[t] = mix4(rd.b, J[t], rd.one_minus_b, recv);
+        const float4 r0 = *reinterpret_cast<const float4 *>(buf + src * kTileCols + c0);
+        const float4 r1 = *reinterpret_cast<const float4 *>(buf + src * kTileCols + c1);
+        I0[t] = mix4(rd.a, I0[t], rd.one_minus_a, r0);
+        I1[t] = mix4(rd.a, I1[t], rd.one_minus_a, r1);
+        J0[t] = mix4(rd.b, J0[t], rd.one_minus_b, r0);
+        J1[t] = mix4(rd.b, J1[t], rd.one_minus_b, r1);
       }
     }
     // no second barrier: the next round writes the other buffer, and a thread can only start
     // the round after that once everybody has passed the next round's barrier.
   }
-  __syncthreads();
+  __syncthreads();  // the last round's reads are done: the tiles can take the results
 
 #pragma unroll
   for (int t = 0; t < R; ++t) {
     const int i = q + t * kRowGroups;
     if (i < n) {
-      *reinterpret_cast<float4 *>(tile_a + i * kTileCols + c) = I[t];
-      if (p.has_y_out) *reinterpret_cast<float4 *>(tile_b + i * kTileCols + c) = J[t];
+      *reinterpret_cast<float4 *>(tile_a + i * kTileCols + c0) = I0[t];
+      *reinterpret_cast<float4 *>(tile_a + i * kTileCols + c1) = I1[t];
+      if (p.has_y_out) {
+        *reinterpret_cast<float4 *>(tile_b + i * kTileCols + c0) = J0[t];
+        *reinterpret_cast<float4 *>(tile_b + i * kTileCols + c1) = J1[t];
+      }
     }
   }
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic writes -> visible to TMA
@@ -229,11 +263,13 @@ static bool make_map(CUtensorMap *map, const float *base, int32_t n, int64_t d, 
 
 template <int R>
 static cudaError_t launch_fused(const CUtensorMap &mxi, const CUtensorMap &myi, const CUtensorMap &mxo,
-                                const CUtensorMap &myo, const FusedArgs &args, int64_t d,
-                                cudaStream_t stream) {
+                                const CUtensorMap &myo, const FusedArgs &args, int64_t d, cudaStream_t stream) {
   const size_t smem = 2 * (size_t)args.n * kTileCols * sizeof(float);
   cudaError_t e = cudaFuncSetAttribute(consensus_fused_kernel<R>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        (int)smem);
+  if (e != cudaSuccess) return e;
+  e = cudaFuncSetAttribute(consensus_fused_kernel<R>, cudaFuncAttributePreferredSharedMemoryCarveout,
+                           cudaSharedmemCarveoutMaxShared);
   if (e != cudaSuccess) return e;
   const int64_t tiles = (d + kTileCols - 1) / kTileCols;
   consensus_fused_kernel<R><<<(unsigned)tiles, kFusedThreads, smem, stream>>>(mxi, myi, mxo, myo, args);
@@ -275,14 +311,12 @@ static ceca_status_t consensus_fused(const float *X, const float *Y, float *Xo, 
   if (!make_map(&myi, args.has_y_in ? Y : X, n, d, ld)) return CECA_ERR_CUDA;
   if (!make_map(&myo, Yo ? Yo : Xo, n, d, ld)) return CECA_ERR_CUDA;
 
-  const int rows_per_thread = (n + kRowGroups - 1) / kRowGroups;  // n <= 256 -> at most 8
+  const int rows_per_thread = (n + kRowGroups - 1) / kRowGroups;  // n <= 256 -> at most 4
   cudaError_t e;
   if (rows_per_thread <= 1)      e = launch_fused<1>(mxi, myi, mxo, myo, args, d, stream);
   else if (rows_per_thread <= 2) e = launch_fused<2>(mxi, myi, mxo, myo, args, d, stream);
   else if (rows_per_thread <= 3) e = launch_fused<3>(mxi, myi, mxo, myo, args, d, stream);
-  else if (rows_per_thread <= 4) e = launch_fused<4>(mxi, myi, mxo, myo, args, d, stream);
-  else if (rows_per_thread <= 6) e = launch_fused<6>(mxi, myi, mxo, myo, args, d, stream);
-  else                           e = launch_fused<8>(mxi, myi, mxo, myo, args, d, stream);
+  else                           e = launch_fused<4>(mxi, myi, mxo, myo, args, d, stream);
   return e == cudaSuccess ? CECA_OK : CECA_ERR_CUDA;
 }
 
