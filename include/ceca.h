@@ -41,7 +41,9 @@ typedef enum {
   CECA_ERR_ALIGNMENT = 3,   /* the fused consensus kernel needs 16-byte aligned rows             */
   CECA_ERR_UNSUPPORTED = 4, /* e.g. in-place aliasing of only one of X/Y, fused path with n > 256 */
   CECA_ERR_WORKSPACE = 5,   /* workspace NULL or smaller than ceca_workspace_bytes says          */
-  CECA_ERR_CUDA = 6         /* a CUDA runtime / driver call failed (launch, copy, map encode)    */
+  CECA_ERR_CUDA = 6,        /* a CUDA runtime / driver call failed (launch, copy, map encode)    */
+  CECA_ERR_STATIC_SCRATCH = 7 /* dsgd_logreg_grad_static: the problem needs more scratch than the
+                                 built-in buffer holds; use dsgd_logreg_grad with a workspace       */
 } ceca_status_t;
 
 /*
@@ -132,6 +134,32 @@ ceca_status_t dsgd_logreg_grad(const float *A, const float *labels, const float 
                                int64_t k, float *G, int32_t n, int32_t m, int64_t d, int64_t ld,
                                ceca_variant_t variant, void *workspace, size_t workspace_bytes,
                                void *stream);
+
+/*
+ * dsgd_logreg_grad for callers that cannot provide a workspace because they cannot allocate device
+ * memory when the gradient is needed: a plug-in inside an application that owns the device heap,
+ * code running where a framework's allocator must not be re-entered, a latency-critical loop that
+ * must stay clear of cudaMalloc.  (The paper has no counterpart to this call; it is a packaging
+ * variant of the one above and computes exactly the same G with the same kernels.)
+ *
+ * The scratch memory is a fixed buffer of dsgd_logreg_grad_static_capacity() bytes (32 MiB) built
+ * into the library; every GPU on which the library is used keeps that much memory from first use
+ * until the process exits.  The call allocates nothing and frees nothing.
+ *   - A problem whose ceca_workspace_bytes(CECA_WS_LOGREG_GRAD, n, m, d) exceeds the capacity is
+ *     rejected with CECA_ERR_STATIC_SCRATCH before anything is launched.
+ *   - The first call on each device looks up the buffer's device address (with that device
+ *     current); make that first call ordinary eager work, before any stream capture is begun.
+ *   - All calls on a device share the one buffer.  Nothing in it needs clearing between calls
+ *     (each call overwrites what it later reads), but two calls that may run on the GPU at the
+ *     same time -- different streams, or different host threads -- race on it: order them.
+ * Arguments, layouts and the other error codes are those of dsgd_logreg_grad.
+ */
+ceca_status_t dsgd_logreg_grad_static(const float *A, const float *labels, const float *X, const float *Y,
+                                      int64_t k, float *G, int32_t n, int32_t m, int64_t d, int64_t ld,
+                                      ceca_variant_t variant, void *stream);
+
+/* Host function.  Size in bytes of the buffer dsgd_logreg_grad_static works in. */
+size_t dsgd_logreg_grad_static_capacity(void);
 
 typedef enum {
   CECA_WS_CONSENSUS_FUSED = 1,    /* ceca_consensus_rounds, fused = 1                      */

@@ -14,7 +14,8 @@ WS_LOGREG_GRAD = 3
 WS_STEP_HOST = 4
 
 EXPORTS = ["ceca_schedule", "ceca_gossip_sgd_step", "ceca_consensus_rounds", "dsgd_logreg_grad",
-           "ceca_workspace_bytes", "ceca_read_status", "ceca_gossip_sgd_step_host", "ceca_status_string"]
+           "ceca_workspace_bytes", "ceca_read_status", "ceca_gossip_sgd_step_host", "ceca_status_string",
+           "dsgd_logreg_grad_static", "dsgd_logreg_grad_static_capacity"]
 
 
 class Round(ctypes.Structure):
@@ -57,6 +58,10 @@ def library():
     lib.dsgd_logreg_grad.argtypes = [vp, vp, vp, vp, i64, vp, i32, i32, i64, i64, i32, vp,
                                      ctypes.c_size_t, vp]
     lib.dsgd_logreg_grad.restype = ctypes.c_int
+    lib.dsgd_logreg_grad_static.argtypes = [vp, vp, vp, vp, i64, vp, i32, i32, i64, i64, i32, vp]
+    lib.dsgd_logreg_grad_static.restype = ctypes.c_int
+    lib.dsgd_logreg_grad_static_capacity.argtypes = []
+    lib.dsgd_logreg_grad_static_capacity.restype = ctypes.c_size_t
     lib.ceca_workspace_bytes.argtypes = [ctypes.c_int, i32, i32, i64]
     lib.ceca_workspace_bytes.restype = ctypes.c_size_t
     lib.ceca_read_status.argtypes = [vp, ctypes.POINTER(i32), vp]
@@ -167,6 +172,33 @@ def dsgd_logreg_grad(A, labels, X, Y, k, variant, G, workspace, stream=None):
                                     _ptr(workspace), ws_bytes, _stream(stream))
     _check(st, "dsgd_logreg_grad")
     return G
+
+
+def dsgd_logreg_grad_static(A, labels, X, Y, k, variant, G, stream=None):
+    """dsgd_logreg_grad without a workspace argument, for callers that cannot allocate device memory
+    (no allocator at hand, or none that may be called at that point): the scratch space is a fixed
+    32 MiB buffer inside the library.  Larger problems raise CecaError (status 7).  Calls on one
+    device share that buffer, so they must not overlap on the GPU."""
+    import torch
+    if A.dtype != torch.float32 or A.dim() != 3 or not A.is_contiguous() or not A.is_cuda:
+        raise ValueError("A must be a contiguous 3-D float32 device tensor")
+    n, m, d = A.shape
+    if labels.dtype != torch.float32 or tuple(labels.shape) != (n, m) or not labels.is_contiguous():
+        raise ValueError("labels must be a contiguous float32 [n, m] tensor")
+    _, dx, ld = _matrix(X, "X", n)
+    if dx != d:
+        raise ValueError("X must have d columns")
+    for t, name in ((Y, "Y"), (G, "G")):
+        if t is not None and _matrix(t, name, n) != (n, d, ld):
+            raise ValueError("%s must have the shape and row stride of X" % name)
+    st = library().dsgd_logreg_grad_static(_ptr(A), _ptr(labels), _ptr(X), _ptr(Y), k, _ptr(G), n, m, d, ld,
+                                           variant, _stream(stream))
+    _check(st, "dsgd_logreg_grad_static")
+    return G
+
+
+def dsgd_logreg_grad_static_capacity():
+    return int(library().dsgd_logreg_grad_static_capacity())
 
 
 def ceca_workspace_bytes(kind, n, m, d):

@@ -16,6 +16,7 @@
 #include <cuda_runtime.h>
 
 #include <cstdint>
+#include <mutex>
 
 #include "ceca.h"
 #include "plan.h"
@@ -228,6 +229,96 @@ extern "C" ceca_status_t dsgd_logreg_grad(const float *A, const float *labels, c
   }
   const int64_t warps = (int64_t)n * m;
   const int64_t blocks1 = (warps * 32 + 255) / 256;
+  const int64_t blocks2 = ((int64_t)n * d + 255) / 256;
+  if (blocks1 > 0x7fffffffLL || blocks2 > 0x7fffffffLL) return CECA_ERR_UNSUPPORTED;
+  logreg_coef_kernel<<<(unsigned)blocks1, 256, 0, stream>>>(A, labels, Z, coef, n, m, d, ld, inv_m);
+  if (cudaGetLastError() != cudaSuccess) return CECA_ERR_CUDA;
+  logreg_accum_kernel<<<(unsigned)blocks2, 256, 0, stream>>>(A, coef, G, n, m, d, ld);
+  return cudaGetLastError() == cudaSuccess ? CECA_OK : CECA_ERR_CUDA;
+}
+
+// ---- the same gradient for callers that cannot hand over a workspace ---------------------------
+//
+// Some callers have no way to get device memory at the moment they need the gradient: a plug-in
+// whose host application owns the whole device heap, code that runs while a framework's caching
+// allocator must not be re-entered, or a latency-critical loop in which cudaMalloc (which can
+// synchronise the whole device) is off limits.  For them the partial sums and coefficients live
+// in the fixed buffer below, which is part of the loaded module: every GPU on which this library
+// is used holds these bytes from the first use until the process exits.
+namespace ceca {
+
+constexpr size_t kStaticScratchBytes = (size_t)32 << 20;  // 32 MiB: enough for n=63, m=2000, d=4096
+static __device__ __align__(256) unsigned char g_logreg_scratch[kStaticScratchBytes];
+
+constexpr int kMaxDevices = 64;
+static std::mutex g_scratch_mutex;
+static void *g_scratch_ptr[kMaxDevices];  // device address of g_logreg_scratch, per device ordinal
+
+// In host code `g_logreg_scratch` is only a handle; the address a kernel can use has to be asked
+// for, once per device, while that device is current.
+static cudaError_t static_scratch_address(void **out) {
+  int dev = -1;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+  std::lock_guard<std::mutex> lock(g_scratch_mutex);
+  if (!g_scratch_ptr[dev]) {
+    void *ptr = nullptr;
+    e = cudaGetSymbolAddress(&ptr, g_logreg_scratch);
+    if (e != cudaSuccess) return e;
+    g_scratch_ptr[dev] = ptr;
+  }
+  *out = g_scratch_ptr[dev];
+  return cudaSuccess;
+}
+
+}  // namespace ceca
+
+extern "C" size_t dsgd_logreg_grad_static_capacity(void) { return ceca::kStaticScratchBytes; }
+
+extern "C" ceca_status_t dsgd_logreg_grad_static(const float *A, const float *labels, const float *X, const float *Y,
+                                                 int64_t k, float *G, int32_t n, int32_t m, int64_t d, int64_t ld,
+                                                 ceca_variant_t variant, void *stream_) {
+  using namespace ceca;
+  if (!A || !labels || !X || !G || n < 1 || m < 1 || d < 1 || ld < d) return CECA_ERR_INVALID_ARG;
+  Plan plan;
+  ceca_status_t st = make_plan(n, variant, k, &plan);
+  if (st != CECA_OK) return st;
+  const float *Z = plan.rd.payload ? Y : X;
+  if (!Z) return CECA_ERR_INVALID_ARG;
+  if (logreg_workspace_bytes(n, m, d) > kStaticScratchBytes) return CECA_ERR_STATIC_SCRATCH;  // nothing launched
+  void *scratch = nullptr;
+  if (static_scratch_address(&scratch) != cudaSuccess) return CECA_ERR_CUDA;
+
+  // From here on: the launches of dsgd_logreg_grad, with the built-in buffer as the workspace.
+  // Nothing in it has to start at zero: every partial sum and every coefficient that is read has
+  // been written earlier in the same call.
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  const float inv_m = (float)(1.0 / (double)m);
+  const int32_t P = logreg_sample_blocks(n, m);
+  float *partial = static_cast<float *>(scratch);
+  const size_t partial_bytes = (((size_t)n * P * d * sizeof(float) + 255) / 256) * 256;
+  float *coef = reinterpret_cast<float *>(static_cast<char *>(scratch) + partial_bytes);
+  const bool fast = (d % 4 == 0) && (ld % 4 == 0) && d <= (int64_t)kLrThreads * 4 * kLrMaxVpt && aligned16(A) &&
+                    aligned16(Z) && aligned16(G) && n <= 65535;
+  if (fast) {
+    LogregArgs a;
+    a.A = A; a.labels = labels; a.Z = Z; a.partial = partial;
+    a.d = d; a.ld = ld; a.n = n; a.m = m; a.P = P;
+    a.samples_per_block = (m + P - 1) / P;
+    a.inv_m = inv_m;
+    const dim3 grid((unsigned)P, (unsigned)n);
+    const int64_t groups = (d / 4 + kLrThreads - 1) / kLrThreads;
+    if (groups <= 1)      logreg_fused_kernel<1><<<grid, kLrThreads, 0, stream>>>(a);
+    else if (groups <= 2) logreg_fused_kernel<2><<<grid, kLrThreads, 0, stream>>>(a);
+    else if (groups <= 4) logreg_fused_kernel<4><<<grid, kLrThreads, 0, stream>>>(a);
+    else                  logreg_fused_kernel<8><<<grid, kLrThreads, 0, stream>>>(a);
+    if (cudaGetLastError() != cudaSuccess) return CECA_ERR_CUDA;
+    const int64_t work = (int64_t)n * (d / 4);
+    logreg_reduce_kernel<<<(unsigned)((work + 255) / 256), 256, 0, stream>>>(partial, G, n, P, d, ld);
+    return cudaGetLastError() == cudaSuccess ? CECA_OK : CECA_ERR_CUDA;
+  }
+  const int64_t blocks1 = ((int64_t)n * m * 32 + 255) / 256;
   const int64_t blocks2 = ((int64_t)n * d + 255) / 256;
   if (blocks1 > 0x7fffffffLL || blocks2 > 0x7fffffffLL) return CECA_ERR_UNSUPPORTED;
   logreg_coef_kernel<<<(unsigned)blocks1, 256, 0, stream>>>(A, labels, Z, coef, n, m, d, ld, inv_m);

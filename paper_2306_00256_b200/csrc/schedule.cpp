@@ -99,6 +99,7 @@ extern "C" const char *ceca_status_string(ceca_status_t status) {
     case CECA_ERR_UNSUPPORTED: return "unsupported combination of arguments";
     case CECA_ERR_WORKSPACE: return "workspace missing or too small";
     case CECA_ERR_CUDA: return "CUDA call failed";
+    case CECA_ERR_STATIC_SCRATCH: return "problem too large for the built-in scratch buffer";
   }
   return "unknown status";
 }
