@@ -49,10 +49,13 @@ FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
 # capture summarised under profiles/ (None until captured, or once the kernel has changed since).
 NCU_TRAFFIC_BYTES_PER_LAUNCH = {
-    # 19.75 B per agent-parameter measured on step_small (2.5167 GB read + 1.6243 GB written for
+    # 19.76 B per agent-parameter measured on step_small (2.5166 GB read + 1.6263 GB written for
     # 100 x 2,097,152 units); traffic is proportional to the units, scaled here to n*d of each workload
-    "step_small": 4.141e9,
-    "resnet50_step": 19.746 * 100 * 25_557_032,
+    "step_small": 4.143e9,
+    "resnet50_step": 19.755 * 100 * 25_557_032,
+    "consensus_fused": 1.165e9,
+    "consensus_rounds": 10.56e9,
+    "logreg_grad": 2.0736e9 + 29.9e6,
 }
 
 
@@ -304,7 +307,8 @@ def bench_consensus(args, wl, device, dist):
     peak, which = measured_peak()
     per_elem = 12 if fused else (16 * tau - 4)   # fused: X in, X and Y out; per round: 16 B (12 B in round 0)
     achieved = per_elem * n * d / (total_ms / args.steps * 1e-3) / 1e9
-    roof = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak, "traffic": None,
+    roof = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+            "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH.get(args.workload),
             "kernel": "consensus_fused_kernel" if fused else "step_walk_kernel<float4, no gradient> x tau",
             "peak_source": "of " + which}
     launches = args.steps * (1 if fused else tau)
@@ -343,7 +347,8 @@ def bench_logreg(args, wl, device, dist):
     grad_ms = sum(ev[2 * s].elapsed_time(ev[2 * s + 1]) for s in range(args.steps)) / args.steps
     peak, which = measured_peak()
     achieved = (4 * n * m * d + 8 * n * d + 4 * n * m) / (grad_ms * 1e-3) / 1e9
-    roof = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak, "traffic": None,
+    roof = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+            "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH.get(args.workload),
             "kernel": "logreg_fused_kernel + logreg_reduce_kernel", "peak_source": "of " + which, "avg_launch_ms": grad_ms}
     return total_ms, 3 * args.steps, roof, clocks, {"m": m, "l2": "A is 2.06 GB, larger than L2"}
 
