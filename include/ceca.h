@@ -136,6 +136,19 @@ ceca_status_t dsgd_logreg_grad(const float *A, const float *labels, const float 
                                void *stream);
 
 /*
+ * Per-agent least-squares gradient, the paper's convex workload (Sec. 5 "DSGD: least-squares
+ * problem"): f_i(w) = 1/2 ||A_i w - b_i||^2 and the stochastic gradient is
+ *   G[i, :] = A_i^T (A_i z_i - b_i) + eps_i
+ * evaluated at the model Algorithm 1 selects in iteration k (z = X if delta_r = 1, else Y).
+ * A: device, n x m x d fp32, dense;  B: device, n x m fp32 (the measurements b_i);
+ * noise: device, n x d with leading dimension ld, the caller's draw of eps (may be NULL = no noise);
+ * X, Y, G, workspace, stream and the error codes: as for dsgd_logreg_grad (same workspace size).
+ */
+ceca_status_t dsgd_lsq_grad(const float *A, const float *B, const float *X, const float *Y, const float *noise,
+                            int64_t k, float *G, int32_t n, int32_t m, int64_t d, int64_t ld,
+                            ceca_variant_t variant, void *workspace, size_t workspace_bytes, void *stream);
+
+/*
  * dsgd_logreg_grad for callers that cannot provide a workspace because they cannot allocate device
  * memory when the gradient is needed: a plug-in inside an application that owns the device heap,
  * code running where a framework's allocator must not be re-entered, a latency-critical loop that
@@ -164,7 +177,7 @@ size_t dsgd_logreg_grad_static_capacity(void);
 typedef enum {
   CECA_WS_CONSENSUS_FUSED = 1,    /* ceca_consensus_rounds, fused = 1                      */
   CECA_WS_CONSENSUS_UNFUSED = 2,  /* ceca_consensus_rounds, fused = 0 with Y_out == NULL   */
-  CECA_WS_LOGREG_GRAD = 3,        /* dsgd_logreg_grad                                      */
+  CECA_WS_LOGREG_GRAD = 3,        /* dsgd_logreg_grad and dsgd_lsq_grad                    */
   CECA_WS_STEP_HOST = 4           /* ceca_gossip_sgd_step_host: the smallest useful size   */
 } ceca_workspace_kind_t;
 

@@ -52,6 +52,8 @@ def lib():
                                                ctypes.c_int64, ctypes.c_int32]
         _lib.ceca_oracle_logreg_grad.argtypes = [dp, dp, dp, dp, ctypes.c_int64, dp, ctypes.c_int32,
                                                  ctypes.c_int32, ctypes.c_int64]
+        _lib.ceca_oracle_lsq_grad.argtypes = [dp, dp, dp, dp, dp, ctypes.c_int64, dp, ctypes.c_int32,
+                                              ctypes.c_int32, ctypes.c_int64]
         _lib.ceca_oracle_logreg_loss.argtypes = [dp, dp, dp, dp, ctypes.c_int32, ctypes.c_int32,
                                                  ctypes.c_int64]
     return _lib
@@ -119,6 +121,17 @@ def logreg_loss(A, labels, W):
     out = np.empty(n, dtype=np.float64)
     _check(lib().ceca_oracle_logreg_loss(_dp(A), _dp(labels), _dp(W), _dp(out), n, m, d))
     return out
+
+
+def lsq_grad(A, B, X, Y, k, noise=None):
+    """Per-agent least-squares gradient A_i^T (A_i z_i - b_i) (+ noise) at the model iteration k selects."""
+    A, B, X, Y = _f64(A), _f64(B), _f64(X), _f64(Y)
+    n, m, d = A.shape
+    N = None if noise is None else _f64(noise)
+    G = np.empty((n, d), dtype=np.float64)
+    _check(lib().ceca_oracle_lsq_grad(_dp(A), _dp(B), _dp(X), _dp(Y), None if N is None else _dp(N), k, _dp(G),
+                                      n, m, d))
+    return G
 
 
 def set_threads(t):

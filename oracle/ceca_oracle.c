@@ -15,6 +15,7 @@
  *   - a CECA round = the same update with gamma = 0 . Sec. 3.1 "Main recursions", Algorithm 2
  *   - logistic-regression gradient .................. NOT in the paper (workload chosen by the
  *                                                     benchmark); pinned by calculus only.
+ *   - least-squares gradient ........................ Sec. 5 "DSGD: least-squares problem"
  *
  * Indices are 0-based here.  The paper's agents are 1..n with a mod that maps into
  * {1..n}; paper agent p is index p-1, so a paper-odd agent has an even index.
@@ -235,6 +236,34 @@ int ceca_oracle_logreg_loss(const double *A, const double *labels, const double 
       acc += v > 0 ? v + log1p(exp(-v)) : log1p(exp(v));
     }
     loss[i] = acc / (double)m;
+  }
+  return ORACLE_OK;
+}
+
+/*
+ * Per-agent least-squares gradient, Sec. 5 "DSGD: least-squares problem":
+ *   f_i(w) = (1/2) ||A_i w - b_i||^2,   stochastic gradient = A_i^T (A_i w - b_i) + eps_i,
+ * evaluated at w = z_i, the model Algorithm 1 selects in iteration k.  The noise eps (n x d, may be
+ * NULL) is an input: the caller draws it.  A is n x m x d, B is n x m.
+ */
+int ceca_oracle_lsq_grad(const double *A, const double *B, const double *X, const double *Y,
+                         const double *noise, int64_t k, double *G, int32_t n, int32_t m, int64_t d) {
+  if (!A || !B || !X || !Y || !G || m < 1 || d < 1) return ORACLE_ERR_ARG;
+  oracle_round_t rd;
+  int rc = ceca_oracle_round(n, k, &rd);
+  if (rc) return rc;
+  const double *Z = rd.payload == 0 ? X : Y;
+#pragma omp parallel for schedule(static)
+  for (int32_t i = 0; i < n; i++) {
+    const double *w = Z + (int64_t)i * d;
+    double *g = G + (int64_t)i * d;
+    for (int64_t c = 0; c < d; c++) g[c] = noise ? noise[(int64_t)i * d + c] : 0.0;
+    for (int32_t s = 0; s < m; s++) {
+      const double *a_s = A + ((int64_t)i * m + s) * d;
+      double resid = -B[(int64_t)i * m + s];
+      for (int64_t c = 0; c < d; c++) resid += a_s[c] * w[c];
+      for (int64_t c = 0; c < d; c++) g[c] += resid * a_s[c];
+    }
   }
   return ORACLE_OK;
 }

@@ -9,10 +9,10 @@ from .binding import (CECA_1P, CECA_2P, CecaError, Round, WS_CONSENSUS_FUSED, WS
                       WS_LOGREG_GRAD, WS_STEP_HOST, ceca_consensus_rounds, ceca_gossip_sgd_step,
                       ceca_gossip_sgd_step_host, ceca_read_status, ceca_schedule, ceca_status_string,
                       ceca_workspace_bytes, dsgd_logreg_grad, dsgd_logreg_grad_static,
-                      dsgd_logreg_grad_static_capacity, library, library_path)
+                      dsgd_logreg_grad_static_capacity, dsgd_lsq_grad, library, library_path)
 
 __all__ = ["CECA_1P", "CECA_2P", "CecaError", "Round", "WS_CONSENSUS_FUSED", "WS_CONSENSUS_UNFUSED",
            "WS_LOGREG_GRAD", "WS_STEP_HOST", "ceca_consensus_rounds", "ceca_gossip_sgd_step",
            "ceca_gossip_sgd_step_host", "ceca_read_status", "ceca_schedule", "ceca_status_string",
            "ceca_workspace_bytes", "dsgd_logreg_grad", "dsgd_logreg_grad_static",
-           "dsgd_logreg_grad_static_capacity", "library", "library_path"]
+           "dsgd_logreg_grad_static_capacity", "dsgd_lsq_grad", "library", "library_path"]

@@ -15,7 +15,7 @@ WS_STEP_HOST = 4
 
 EXPORTS = ["ceca_schedule", "ceca_gossip_sgd_step", "ceca_consensus_rounds", "dsgd_logreg_grad",
            "ceca_workspace_bytes", "ceca_read_status", "ceca_gossip_sgd_step_host", "ceca_status_string",
-           "dsgd_logreg_grad_static", "dsgd_logreg_grad_static_capacity"]
+           "dsgd_logreg_grad_static", "dsgd_logreg_grad_static_capacity", "dsgd_lsq_grad"]
 
 
 class Round(ctypes.Structure):
@@ -58,6 +58,8 @@ def library():
     lib.dsgd_logreg_grad.argtypes = [vp, vp, vp, vp, i64, vp, i32, i32, i64, i64, i32, vp,
                                      ctypes.c_size_t, vp]
     lib.dsgd_logreg_grad.restype = ctypes.c_int
+    lib.dsgd_lsq_grad.argtypes = [vp, vp, vp, vp, vp, i64, vp, i32, i32, i64, i64, i32, vp, ctypes.c_size_t, vp]
+    lib.dsgd_lsq_grad.restype = ctypes.c_int
     lib.dsgd_logreg_grad_static.argtypes = [vp, vp, vp, vp, i64, vp, i32, i32, i64, i64, i32, vp]
     lib.dsgd_logreg_grad_static.restype = ctypes.c_int
     lib.dsgd_logreg_grad_static_capacity.argtypes = []
@@ -171,6 +173,27 @@ def dsgd_logreg_grad(A, labels, X, Y, k, variant, G, workspace, stream=None):
     st = library().dsgd_logreg_grad(_ptr(A), _ptr(labels), _ptr(X), _ptr(Y), k, _ptr(G), n, m, d, ld, variant,
                                     _ptr(workspace), ws_bytes, _stream(stream))
     _check(st, "dsgd_logreg_grad")
+    return G
+
+
+def dsgd_lsq_grad(A, B, X, Y, k, variant, G, workspace, noise=None, stream=None):
+    """Per-agent least-squares gradient A_i^T (A_i z_i - b_i) (+ noise) at the model iteration k selects."""
+    import torch
+    if A.dtype != torch.float32 or A.dim() != 3 or not A.is_contiguous() or not A.is_cuda:
+        raise ValueError("A must be a contiguous 3-D float32 device tensor")
+    n, m, d = A.shape
+    if B.dtype != torch.float32 or tuple(B.shape) != (n, m) or not B.is_contiguous():
+        raise ValueError("B must be a contiguous float32 [n, m] tensor")
+    _, dx, ld = _matrix(X, "X", n)
+    if dx != d:
+        raise ValueError("X must have d columns")
+    for t, name in ((Y, "Y"), (G, "G"), (noise, "noise")):
+        if t is not None and _matrix(t, name, n) != (n, d, ld):
+            raise ValueError("%s must have the shape and row stride of X" % name)
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    st = library().dsgd_lsq_grad(_ptr(A), _ptr(B), _ptr(X), _ptr(Y), _ptr(noise), k, _ptr(G), n, m, d, ld, variant,
+                                 _ptr(workspace), ws_bytes, _stream(stream))
+    _check(st, "dsgd_lsq_grad")
     return G
 
 

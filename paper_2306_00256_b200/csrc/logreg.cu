@@ -1,6 +1,10 @@
-// Per-agent logistic-regression gradient (the e^(k) of Algorithm 1 for the synthetic
-// classification workloads; the loss itself is not from the paper):
-//   G[i, :] = -(1/m) sum_s l_s sigma(-l_s <a_s, z_i>) a_s,   z = X if delta_r = 1 else Y.
+// Per-agent gradients e^(k) of Algorithm 1 for two data-fitting losses over local samples (a_s, t_s):
+//   logistic (synthetic classification workloads; this loss is not from the paper)
+//     G[i, :] = -(1/m) sum_s l_s sigma(-l_s <a_s, z_i>) a_s
+//   least squares (Sec. 5 "DSGD: least-squares problem": f_i(w) = 1/2 ||A_i w - b_i||^2)
+//     G[i, :] = sum_s (<a_s, z_i> - b_s) a_s  (+ eps_i, the caller's gradient noise)
+// with z = X if delta_r = 1 else Y.  Both are "coefficient per sample times the sample", so they
+// share the kernels below; only the coefficient differs.
 //
 // Main path (d a multiple of 4, d <= 8192, 16-byte aligned rows): A is read exactly once.  A CTA
 // takes one agent and a block of its samples; each thread keeps its slice of z_i and of the
@@ -37,6 +41,16 @@ static inline int32_t logreg_sample_blocks(int32_t n, int32_t m) {
   return (int32_t)p;
 }
 
+constexpr int kLossLogistic = 0;
+constexpr int kLossSquare = 1;
+
+// The per-sample coefficient c_s such that the gradient is sum_s c_s a_s; t = <a_s, z_i>.
+template <int LOSS>
+__device__ __forceinline__ float sample_coef(float target, float t, float inv_m) {
+  if (LOSS == kLossLogistic) return -target * inv_m / (1.f + expf(target * t));  // -l sigma(-l t) / m
+  return t - target;                                                             // residual a.z - b
+}
+
 struct LogregArgs {
   const float *A, *labels, *Z;
   float *partial;   // [n][P][d]
@@ -49,7 +63,7 @@ __device__ __forceinline__ float dot4(float4 a, float4 b) {
   return fmaf(a.x, b.x, fmaf(a.y, b.y, fmaf(a.z, b.z, a.w * b.w)));
 }
 
-template <int VPT>
+template <int VPT, int LOSS>
 __global__ void __launch_bounds__(kLrThreads) logreg_fused_kernel(const LogregArgs p) {
   __shared__ float4 red[2][kLrWarps];
   const int i = blockIdx.y;
@@ -110,8 +124,7 @@ __global__ void __launch_bounds__(kLrThreads) logreg_fused_kernel(const LogregAr
     for (int jj = 0; jj < kLrSamples; ++jj) {
       float coef = 0.f;
       if (s + jj < s_end) {
-        const float l = __ldg(l_agent + s + jj);
-        coef = -l * p.inv_m / (1.f + expf(l * margin[jj]));  // -l sigma(-l t) / m
+        coef = sample_coef<LOSS>(__ldg(l_agent + s + jj), margin[jj], p.inv_m);
       }
 #pragma unroll
       for (int j = 0; j < VPT; ++j) {
@@ -130,9 +143,9 @@ __global__ void __launch_bounds__(kLrThreads) logreg_fused_kernel(const LogregAr
   }
 }
 
-// G[i, c..c+3] = sum over the P partials, in block order.
-__global__ void __launch_bounds__(256) logreg_reduce_kernel(const float *partial, float *G, int32_t n, int32_t P,
-                                                            int64_t d, int64_t ld) {
+// G[i, c..c+3] = sum over the P partials, in block order (+ the caller's noise, if any).
+__global__ void __launch_bounds__(256) logreg_reduce_kernel(const float *partial, const float *noise, float *G,
+                                                            int32_t n, int32_t P, int64_t d, int64_t ld) {
   const int64_t d4 = d >> 2;
   const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (idx >= (int64_t)n * d4) return;
@@ -143,10 +156,15 @@ __global__ void __launch_bounds__(256) logreg_reduce_kernel(const float *partial
     const float4 v = *reinterpret_cast<const float4 *>(src + (int64_t)b * d);
     s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
   }
+  if (noise) {
+    const float4 e = *reinterpret_cast<const float4 *>(noise + i * ld + cg * 4);
+    s.x += e.x; s.y += e.y; s.z += e.z; s.w += e.w;
+  }
   *reinterpret_cast<float4 *>(G + i * ld + cg * 4) = s;
 }
 
 // ---- fallback: any d, any alignment ---------------------------------------------------------
+template <int LOSS>
 __global__ void __launch_bounds__(256) logreg_coef_kernel(const float *A, const float *labels, const float *Z,
                                                           float *coef, int32_t n, int32_t m, int64_t d, int64_t ld,
                                                           float inv_m) {
@@ -160,14 +178,11 @@ __global__ void __launch_bounds__(256) logreg_coef_kernel(const float *A, const 
   for (int64_t c = lane; c < d; c += 32) t = fmaf(row[c], z[c], t);
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
-  if (lane == 0) {
-    const float l = labels[sample];
-    coef[sample] = -l * inv_m / (1.f + expf(l * t));
-  }
+  if (lane == 0) coef[sample] = sample_coef<LOSS>(labels[sample], t, inv_m);
 }
 
-__global__ void __launch_bounds__(256) logreg_accum_kernel(const float *A, const float *coef, float *G, int32_t n,
-                                                           int32_t m, int64_t d, int64_t ld) {
+__global__ void __launch_bounds__(256) logreg_accum_kernel(const float *A, const float *coef, const float *noise,
+                                                           float *G, int32_t n, int32_t m, int64_t d, int64_t ld) {
   const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (idx >= (int64_t)n * d) return;
   const int64_t i = idx / d, c = idx - i * d;
@@ -175,6 +190,7 @@ __global__ void __launch_bounds__(256) logreg_accum_kernel(const float *A, const
   const float *cf = coef + i * m;
   float g = 0.f;
   for (int32_t s = 0; s < m; ++s) g = fmaf(cf[s], col[(int64_t)s * d], g);
+  if (noise) g += noise[i * ld + c];
   G[i * ld + c] = g;
 }
 
@@ -186,55 +202,84 @@ size_t logreg_workspace_bytes(int32_t n, int32_t m, int64_t d) {
   return ((partial + 255) / 256) * 256 + ((coef + 255) / 256) * 256;
 }
 
-}  // namespace ceca
-
-extern "C" ceca_status_t dsgd_logreg_grad(const float *A, const float *labels, const float *X, const float *Y,
-                                          int64_t k, float *G, int32_t n, int32_t m, int64_t d, int64_t ld,
-                                          ceca_variant_t variant, void *workspace, size_t workspace_bytes,
-                                          void *stream_) {
-  using namespace ceca;
-  if (!A || !labels || !X || !G || n < 1 || m < 1 || d < 1 || ld < d) return CECA_ERR_INVALID_ARG;
-  Plan plan;
-  ceca_status_t st = make_plan(n, variant, k, &plan);
-  if (st != CECA_OK) return st;
-  const float *Z = plan.rd.payload ? Y : X;
-  if (!Z) return CECA_ERR_INVALID_ARG;
-  if (!workspace || workspace_bytes < logreg_workspace_bytes(n, m, d) || !aligned16(workspace))
-    return CECA_ERR_WORKSPACE;
-  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+// Enqueues the gradient kernels with `scratch` (>= logreg_workspace_bytes) as working memory.
+// Nothing in the scratch has to start at zero: every partial sum and every coefficient that is read
+// has been written earlier in the same call.
+template <int LOSS>
+static ceca_status_t enqueue_grad(const float *A, const float *targets, const float *Z, const float *noise, float *G,
+                                  int32_t n, int32_t m, int64_t d, int64_t ld, void *scratch, cudaStream_t stream) {
   const float inv_m = (float)(1.0 / (double)m);
   const int32_t P = logreg_sample_blocks(n, m);
-  float *partial = static_cast<float *>(workspace);
+  float *partial = static_cast<float *>(scratch);
   const size_t partial_bytes = (((size_t)n * P * d * sizeof(float) + 255) / 256) * 256;
-  float *coef = reinterpret_cast<float *>(static_cast<char *>(workspace) + partial_bytes);
-
+  float *coef = reinterpret_cast<float *>(static_cast<char *>(scratch) + partial_bytes);
   const bool fast = (d % 4 == 0) && (ld % 4 == 0) && d <= (int64_t)kLrThreads * 4 * kLrMaxVpt && aligned16(A) &&
-                    aligned16(Z) && aligned16(G) && n <= 65535;
+                    aligned16(Z) && aligned16(G) && (!noise || aligned16(noise)) && n <= 65535;
   if (fast) {
     LogregArgs a;
-    a.A = A; a.labels = labels; a.Z = Z; a.partial = partial;
+    a.A = A; a.labels = targets; a.Z = Z; a.partial = partial;
     a.d = d; a.ld = ld; a.n = n; a.m = m; a.P = P;
     a.samples_per_block = (m + P - 1) / P;
     a.inv_m = inv_m;
     const dim3 grid((unsigned)P, (unsigned)n);
     const int64_t groups = (d / 4 + kLrThreads - 1) / kLrThreads;
-    if (groups <= 1)      logreg_fused_kernel<1><<<grid, kLrThreads, 0, stream>>>(a);
-    else if (groups <= 2) logreg_fused_kernel<2><<<grid, kLrThreads, 0, stream>>>(a);
-    else if (groups <= 4) logreg_fused_kernel<4><<<grid, kLrThreads, 0, stream>>>(a);
-    else                  logreg_fused_kernel<8><<<grid, kLrThreads, 0, stream>>>(a);
+    if (groups <= 1)      logreg_fused_kernel<1, LOSS><<<grid, kLrThreads, 0, stream>>>(a);
+    else if (groups <= 2) logreg_fused_kernel<2, LOSS><<<grid, kLrThreads, 0, stream>>>(a);
+    else if (groups <= 4) logreg_fused_kernel<4, LOSS><<<grid, kLrThreads, 0, stream>>>(a);
+    else                  logreg_fused_kernel<8, LOSS><<<grid, kLrThreads, 0, stream>>>(a);
     if (cudaGetLastError() != cudaSuccess) return CECA_ERR_CUDA;
     const int64_t work = (int64_t)n * (d / 4);
-    logreg_reduce_kernel<<<(unsigned)((work + 255) / 256), 256, 0, stream>>>(partial, G, n, P, d, ld);
+    logreg_reduce_kernel<<<(unsigned)((work + 255) / 256), 256, 0, stream>>>(partial, noise, G, n, P, d, ld);
     return cudaGetLastError() == cudaSuccess ? CECA_OK : CECA_ERR_CUDA;
   }
-  const int64_t warps = (int64_t)n * m;
-  const int64_t blocks1 = (warps * 32 + 255) / 256;
+  const int64_t blocks1 = ((int64_t)n * m * 32 + 255) / 256;
   const int64_t blocks2 = ((int64_t)n * d + 255) / 256;
   if (blocks1 > 0x7fffffffLL || blocks2 > 0x7fffffffLL) return CECA_ERR_UNSUPPORTED;
-  logreg_coef_kernel<<<(unsigned)blocks1, 256, 0, stream>>>(A, labels, Z, coef, n, m, d, ld, inv_m);
+  logreg_coef_kernel<LOSS><<<(unsigned)blocks1, 256, 0, stream>>>(A, targets, Z, coef, n, m, d, ld, inv_m);
   if (cudaGetLastError() != cudaSuccess) return CECA_ERR_CUDA;
-  logreg_accum_kernel<<<(unsigned)blocks2, 256, 0, stream>>>(A, coef, G, n, m, d, ld);
+  logreg_accum_kernel<<<(unsigned)blocks2, 256, 0, stream>>>(A, coef, noise, G, n, m, d, ld);
   return cudaGetLastError() == cudaSuccess ? CECA_OK : CECA_ERR_CUDA;
+}
+
+// Argument checks shared by the gradient entry points; picks z by the round of iteration k.
+static ceca_status_t grad_args(const float *A, const float *targets, const float *X, const float *Y, int64_t k,
+                               const float *G, int32_t n, int32_t m, int64_t d, int64_t ld, ceca_variant_t variant,
+                               const float **Z) {
+  if (!A || !targets || !X || !G || n < 1 || m < 1 || d < 1 || ld < d) return CECA_ERR_INVALID_ARG;
+  Plan plan;
+  ceca_status_t st = make_plan(n, variant, k, &plan);
+  if (st != CECA_OK) return st;
+  *Z = plan.rd.payload ? Y : X;
+  return *Z ? CECA_OK : CECA_ERR_INVALID_ARG;
+}
+
+}  // namespace ceca
+
+extern "C" ceca_status_t dsgd_logreg_grad(const float *A, const float *labels, const float *X, const float *Y,
+                                          int64_t k, float *G, int32_t n, int32_t m, int64_t d, int64_t ld,
+                                          ceca_variant_t variant, void *workspace, size_t workspace_bytes,
+                                          void *stream) {
+  using namespace ceca;
+  const float *Z = nullptr;
+  ceca_status_t st = grad_args(A, labels, X, Y, k, G, n, m, d, ld, variant, &Z);
+  if (st != CECA_OK) return st;
+  if (!workspace || workspace_bytes < logreg_workspace_bytes(n, m, d) || !aligned16(workspace))
+    return CECA_ERR_WORKSPACE;
+  return enqueue_grad<kLossLogistic>(A, labels, Z, nullptr, G, n, m, d, ld, workspace,
+                                     static_cast<cudaStream_t>(stream));
+}
+
+extern "C" ceca_status_t dsgd_lsq_grad(const float *A, const float *B, const float *X, const float *Y,
+                                       const float *noise, int64_t k, float *G, int32_t n, int32_t m, int64_t d,
+                                       int64_t ld, ceca_variant_t variant, void *workspace, size_t workspace_bytes,
+                                       void *stream) {
+  using namespace ceca;
+  const float *Z = nullptr;
+  ceca_status_t st = grad_args(A, B, X, Y, k, G, n, m, d, ld, variant, &Z);
+  if (st != CECA_OK) return st;
+  if (!workspace || workspace_bytes < logreg_workspace_bytes(n, m, d) || !aligned16(workspace))
+    return CECA_ERR_WORKSPACE;
+  return enqueue_grad<kLossSquare>(A, B, Z, noise, G, n, m, d, ld, workspace, static_cast<cudaStream_t>(stream));
 }
 
 // ---- the same gradient for callers that cannot hand over a workspace ---------------------------
@@ -278,51 +323,14 @@ extern "C" size_t dsgd_logreg_grad_static_capacity(void) { return ceca::kStaticS
 
 extern "C" ceca_status_t dsgd_logreg_grad_static(const float *A, const float *labels, const float *X, const float *Y,
                                                  int64_t k, float *G, int32_t n, int32_t m, int64_t d, int64_t ld,
-                                                 ceca_variant_t variant, void *stream_) {
+                                                 ceca_variant_t variant, void *stream) {
   using namespace ceca;
-  if (!A || !labels || !X || !G || n < 1 || m < 1 || d < 1 || ld < d) return CECA_ERR_INVALID_ARG;
-  Plan plan;
-  ceca_status_t st = make_plan(n, variant, k, &plan);
+  const float *Z = nullptr;
+  ceca_status_t st = grad_args(A, labels, X, Y, k, G, n, m, d, ld, variant, &Z);
   if (st != CECA_OK) return st;
-  const float *Z = plan.rd.payload ? Y : X;
-  if (!Z) return CECA_ERR_INVALID_ARG;
   if (logreg_workspace_bytes(n, m, d) > kStaticScratchBytes) return CECA_ERR_STATIC_SCRATCH;  // nothing launched
   void *scratch = nullptr;
   if (static_scratch_address(&scratch) != cudaSuccess) return CECA_ERR_CUDA;
-
-  // From here on: the launches of dsgd_logreg_grad, with the built-in buffer as the workspace.
-  // Nothing in it has to start at zero: every partial sum and every coefficient that is read has
-  // been written earlier in the same call.
-  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
-  const float inv_m = (float)(1.0 / (double)m);
-  const int32_t P = logreg_sample_blocks(n, m);
-  float *partial = static_cast<float *>(scratch);
-  const size_t partial_bytes = (((size_t)n * P * d * sizeof(float) + 255) / 256) * 256;
-  float *coef = reinterpret_cast<float *>(static_cast<char *>(scratch) + partial_bytes);
-  const bool fast = (d % 4 == 0) && (ld % 4 == 0) && d <= (int64_t)kLrThreads * 4 * kLrMaxVpt && aligned16(A) &&
-                    aligned16(Z) && aligned16(G) && n <= 65535;
-  if (fast) {
-    LogregArgs a;
-    a.A = A; a.labels = labels; a.Z = Z; a.partial = partial;
-    a.d = d; a.ld = ld; a.n = n; a.m = m; a.P = P;
-    a.samples_per_block = (m + P - 1) / P;
-    a.inv_m = inv_m;
-    const dim3 grid((unsigned)P, (unsigned)n);
-    const int64_t groups = (d / 4 + kLrThreads - 1) / kLrThreads;
-    if (groups <= 1)      logreg_fused_kernel<1><<<grid, kLrThreads, 0, stream>>>(a);
-    else if (groups <= 2) logreg_fused_kernel<2><<<grid, kLrThreads, 0, stream>>>(a);
-    else if (groups <= 4) logreg_fused_kernel<4><<<grid, kLrThreads, 0, stream>>>(a);
-    else                  logreg_fused_kernel<8><<<grid, kLrThreads, 0, stream>>>(a);
-    if (cudaGetLastError() != cudaSuccess) return CECA_ERR_CUDA;
-    const int64_t work = (int64_t)n * (d / 4);
-    logreg_reduce_kernel<<<(unsigned)((work + 255) / 256), 256, 0, stream>>>(partial, G, n, P, d, ld);
-    return cudaGetLastError() == cudaSuccess ? CECA_OK : CECA_ERR_CUDA;
-  }
-  const int64_t blocks1 = ((int64_t)n * m * 32 + 255) / 256;
-  const int64_t blocks2 = ((int64_t)n * d + 255) / 256;
-  if (blocks1 > 0x7fffffffLL || blocks2 > 0x7fffffffLL) return CECA_ERR_UNSUPPORTED;
-  logreg_coef_kernel<<<(unsigned)blocks1, 256, 0, stream>>>(A, labels, Z, coef, n, m, d, ld, inv_m);
-  if (cudaGetLastError() != cudaSuccess) return CECA_ERR_CUDA;
-  logreg_accum_kernel<<<(unsigned)blocks2, 256, 0, stream>>>(A, coef, G, n, m, d, ld);
-  return cudaGetLastError() == cudaSuccess ? CECA_OK : CECA_ERR_CUDA;
+  return enqueue_grad<kLossLogistic>(A, labels, Z, nullptr, G, n, m, d, ld, scratch,
+                                     static_cast<cudaStream_t>(stream));
 }

@@ -71,3 +71,20 @@ def logreg_problem(n, m, d, seed=0, flip=0.1, hetero_std=0.0, device="cpu"):
         flips = torch.rand(m, generator=gen, device=device) < flip
         labels[i] = torch.where(flips, -clean, clean)
     return a, labels, x_star
+
+
+def lsq_problem(n, m, d, seed=0, sigma_s=0.1, device="cpu"):
+    """Distributed least squares: A_i ~ N(0, I) (m x d per agent), x_star ~ N(0, 1)^d,
+    b_i = A_i x_star + v_i with v_i ~ N(0, sigma_s^2 I).  Returns (A [n, m, d], B [n, m], x_star [d])."""
+    gen = _gen(seed, device)
+    x_star = torch.empty(d, dtype=torch.float32, device=device).normal_(generator=gen)
+    a = torch.empty((n, m, d), dtype=torch.float32, device=device).normal_(generator=gen)
+    v = torch.empty((n, m), dtype=torch.float32, device=device).normal_(std=sigma_s, generator=gen)
+    b = torch.einsum("nmd,d->nm", a, x_star) + v
+    return a, b, x_star
+
+
+def gradient_noise(n, d, k, sigma_n, seed=0, device="cpu"):
+    """The additive gradient noise eps_i ~ N(0, sigma_n^2 I) of iteration k (one draw per agent)."""
+    gen = _gen(7_000_003 * (int(seed) + 1) + int(k), device)
+    return torch.empty((n, d), dtype=torch.float32, device=device).normal_(std=sigma_n, generator=gen)

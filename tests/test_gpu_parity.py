@@ -287,6 +287,73 @@ def test_small_logistic_regression_run(n, variant):
 
 
 # --------------------------------------------------------------------------------------------
+# least-squares gradient and the paper's convex experiment (Sec. 5 "DSGD: least-squares problem")
+# --------------------------------------------------------------------------------------------
+
+def _lsq_tol(a, b, z):
+    """fp32 bound: a length-d dot product per residual, then a length-m sum of residual * feature."""
+    n, m, d = a.shape
+    u = 2.0 ** -24
+    mag = np.einsum("nmd,nd->nm", np.abs(a), np.abs(z)) + np.abs(b)          # size of each residual's terms
+    s = np.einsum("nmd,nm->nd", np.abs(a), mag).max()                         # size of each gradient entry's terms
+    return 4 * u * (np.sqrt(d) + np.sqrt(m)) * s + 1e-7
+
+
+@pytest.mark.parametrize("n,m,d", [(258, 50, 10), (6, 50, 10), (4, 64, 2048), (3, 37, 4096), (5, 20, 12), (2, 7, 1)])
+def test_lsq_grad_matches_oracle(n, m, d):
+    a, b, _ = synth.lsq_problem(n, m, d, seed=n + d, sigma_s=0.1)
+    gen = torch.Generator().manual_seed(3)
+    x = torch.randn(n, d, generator=gen); y = torch.randn(n, d, generator=gen)
+    eps = synth.gradient_noise(n, d, 0, sigma_n=5.0)
+    A, B, X, Y, E = a.to(DEV), b.to(DEV), x.to(DEV), y.to(DEV), eps.to(DEV)
+    ws = torch.empty(ceca.ceca_workspace_bytes(ceca.WS_LOGREG_GRAD, n, m, d) // 4 + 64, dtype=torch.float32, device=DEV)
+    for variant in _variants(n):
+        for k in range(min(_tau(n), 4)):
+            z = y if oracle.round_info(n, k).payload else x
+            tol = _lsq_tol(_np(a), _np(b), _np(z))
+            G = torch.full((n, d), float("nan"), device=DEV)
+            ceca.dsgd_lsq_grad(A, B, X, Y, k, variant, G, ws)
+            want = oracle.lsq_grad(_np(a), _np(b), _np(x), _np(y), k)
+            assert np.abs(_np(G) - want).max() <= tol, (n, m, d, k)
+            ceca.dsgd_lsq_grad(A, B, X, Y, k, variant, G, ws, noise=E)
+            want = oracle.lsq_grad(_np(a), _np(b), _np(x), _np(y), k, noise=_np(eps))
+            assert np.abs(_np(G) - want).max() <= tol + 5e-6, (n, m, d, k)
+
+
+@pytest.mark.parametrize("variant", [ceca.CECA_1P, ceca.CECA_2P])
+def test_least_squares_experiment(variant):
+    """n = 258 agents, d = 10, 50 samples each, sigma_s = 0.1, gradient noise sigma_n = 5, step size 0.02
+    divided by 1.5 every 20 iterations: gradient kernel + fused step on the GPU against the fp64 oracle
+    on the same data and the same noise draws."""
+    n, m, d, iters = 258, 50, 10, 120
+    a, b, x_star = synth.lsq_problem(n, m, d, seed=0, sigma_s=0.1)
+    x0 = torch.randn(n, d, generator=torch.Generator().manual_seed(5))
+    A, B = a.to(DEV), b.to(DEV)
+    X, Y, G = x0.to(DEV), x0.to(DEV), torch.empty(n, d, device=DEV)
+    ws = torch.empty(ceca.ceca_workspace_bytes(ceca.WS_LOGREG_GRAD, n, m, d) // 4 + 64, dtype=torch.float32, device=DEV)
+    ox, oy = _np(x0).astype(np.float64), _np(x0).astype(np.float64)
+    an, bn = _np(a), _np(b)
+    err0 = np.linalg.norm(ox.mean(0) - _np(x_star))
+    gamma = 0.02
+    for k in range(iters):
+        if k and k % 20 == 0:
+            gamma /= 1.5
+        eps = synth.gradient_noise(n, d, k, sigma_n=5.0)
+        ceca.dsgd_lsq_grad(A, B, X, Y, k, variant, G, ws, noise=eps.to(DEV))
+        ceca.ceca_gossip_sgd_step(X, Y, G, gamma, variant, k)
+        og = oracle.lsq_grad(an, bn, ox, oy, k, noise=_np(eps))
+        ox, oy = oracle.step(ox, oy, og, np.float32(gamma), variant, k)
+        # the local problems are contractive at this step size, so rounding does not accumulate
+        # faster than linearly; the scale is what one step moves (gamma |G|) or the state itself
+        scale = max(np.abs(ox).max(), np.abs(oy).max(), float(np.float32(gamma)) * np.abs(og).max())
+        tol = 4e-6 * (k + 1) * scale
+        assert np.abs(_np(X) - ox).max() <= tol, k
+        assert np.abs(_np(Y) - oy).max() <= tol, k
+    err1 = np.linalg.norm(_np(X).astype(np.float64).mean(0) - _np(x_star))
+    assert err1 < 0.2 * err0      # the averaged model has moved most of the way to x*
+
+
+# --------------------------------------------------------------------------------------------
 # host-memory front end
 # --------------------------------------------------------------------------------------------
 

@@ -413,3 +413,31 @@ def test_logreg_uses_the_model_algorithm_1_selects():
     np.testing.assert_array_equal(oracle.logreg_grad(a, lab, x, y, 0), oracle.logreg_grad(a, lab, x, x, 0))
     np.testing.assert_array_equal(oracle.logreg_grad(a, lab, x, y, 1), oracle.logreg_grad(a, lab, y, y, 0))
     np.testing.assert_array_equal(oracle.logreg_grad(a, lab, x, y, 2), oracle.logreg_grad(a, lab, x, x, 0))
+
+
+# ---- least-squares gradient (Sec. 5 "DSGD: least-squares problem") ------------------------------
+
+def test_lsq_gradient_vanishes_at_the_least_squares_solution_and_matches_differences():
+    rng = np.random.default_rng(8)
+    n, m, d = 4, 50, 10
+    a = rng.normal(size=(n, m, d)); b = rng.normal(size=(n, m))
+    # at the minimiser of each f_i (library routine) the gradient is zero
+    w_ls = np.stack([np.linalg.lstsq(a[i], b[i], rcond=None)[0] for i in range(n)])
+    g = oracle.lsq_grad(a, b, w_ls, w_ls, 0)
+    assert np.abs(g).max() < 1e-10
+    # elsewhere it is the derivative of (1/2)||A w - b||^2, and the noise is simply added
+    w = rng.normal(size=(n, d)); eps = rng.normal(size=(n, d))
+    g = oracle.lsq_grad(a, b, w, w, 0)
+    loss = lambda wm: 0.5 * ((np.einsum("nmd,nd->nm", a, wm) - b) ** 2).sum(axis=1)
+    h = 1e-5
+    for i in range(n):
+        for c in range(d):
+            wp, wm = w.copy(), w.copy(); wp[i, c] += h; wm[i, c] -= h
+            assert g[i, c] == pytest.approx((loss(wp)[i] - loss(wm)[i]) / (2 * h), rel=1e-7, abs=1e-7)
+    np.testing.assert_allclose(oracle.lsq_grad(a, b, w, w, 0, noise=eps), g + eps, rtol=0, atol=1e-12)
+    # hand case: one sample, one feature: a (a w - b)
+    assert oracle.lsq_grad([[[3.0]]], [[2.0]], [[1.5]], [[0.0]], 0)[0, 0] == pytest.approx(3.0 * (4.5 - 2.0))
+    # the model is the one Algorithm 1 selects (n = 6: round 1 evaluates at y)
+    a6 = rng.normal(size=(6, 5, 3)); b6 = rng.normal(size=(6, 5)); x6 = rng.normal(size=(6, 3)); y6 = rng.normal(size=(6, 3))
+    np.testing.assert_array_equal(oracle.lsq_grad(a6, b6, x6, y6, 1), oracle.lsq_grad(a6, b6, y6, y6, 0))
+    np.testing.assert_array_equal(oracle.lsq_grad(a6, b6, x6, y6, 2), oracle.lsq_grad(a6, b6, x6, x6, 0))
