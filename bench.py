@@ -43,6 +43,8 @@ WORKLOADS = {
     "consensus_fused": dict(kind="consensus", n=97, d=1 << 20, variant=2, fused=1),
     "consensus_rounds": dict(kind="consensus", n=97, d=1 << 20, variant=2, fused=0),
     "logreg_grad": dict(kind="logreg", n=63, m=2000, d=4096, variant=2, gamma=0.01),
+    # n = 2..128 at d = 4,194,304, both variants where defined: kernel and schedule scaling with n
+    "n_sweep": dict(kind="sweep", n=128, d=4_194_304, variant=2, gamma=0.1),
 }
 
 FALLBACK_HBM_GBS = 6650.0
@@ -353,6 +355,55 @@ def bench_logreg(args, wl, device, dist):
     return total_ms, 3 * args.steps, roof, clocks, {"m": m, "l2": "A is 2.06 GB, larger than L2"}
 
 
+def bench_sweep(args, wl, device, dist):
+    """One full CECA cycle (tau fused steps, in place) per n and variant; also the host schedule call."""
+    import torch
+    import paper_2306_00256_b200 as ceca
+    import synthetic_inputs as synth
+    n_max, d, gamma = wl["n"], wl["d"], wl["gamma"]
+    X, Y, G = synth.step_inputs(n_max, d, seed=0, x_std=0.01, g_std=0.01, device=device)
+    stream = torch.cuda.current_stream()
+    peak, which = measured_peak()
+    rows, launches, total_ms, total_units = [], 0, 0.0, 0
+    sampler = ClockSampler(torch.cuda.current_device())
+    sampler.start()
+    for n in range(2, n_max + 1):
+        for variant in (2, 1):
+            if variant == 1 and n % 2:
+                continue
+            tau = ceca.ceca_schedule(n, variant, 0, peers=False)[0].tau
+            t0 = time.perf_counter()
+            for k in range(tau):
+                ceca.ceca_schedule(n, variant, k)
+            sched_us = (time.perf_counter() - t0) / tau * 1e6
+            x, y, g = X[:n], Y[:n], G[:n]
+            for k in range(tau):  # warm-up cycle
+                ceca.ceca_gossip_sgd_step(x, y, g, gamma, variant, k)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            e0.record(stream)
+            for rep in range(args.steps):
+                for k in range(tau):
+                    ceca.ceca_gossip_sgd_step(x, y, g, gamma, variant, k)
+            e1.record(stream)
+            torch.cuda.synchronize()
+            ms = e0.elapsed_time(e1) / (args.steps * tau)
+            gbs = (20 * tau - 4) / tau * n * d / (ms * 1e-3) / 1e9
+            rows.append({"n": n, "variant": "2P" if variant == 2 else "1P", "tau": tau, "ms_per_step": round(ms, 4),
+                         "updates_per_s": n * d / (ms * 1e-3), "gbs": round(gbs, 1), "frac": round(gbs / peak, 3),
+                         "schedule_us": round(sched_us, 2)})
+            launches += args.steps * tau
+            total_ms += e0.elapsed_time(e1)
+            total_units += args.steps * tau * n * d
+    clocks = sampler.stop()
+    fr = sorted(r["frac"] for r in rows)
+    roof = {"bound": "hbm", "achieved": fr[len(fr) // 2] * peak, "peak": peak, "unit": "GB/s", "frac": fr[len(fr) // 2],
+            "traffic": None, "kernel": "step_walk_kernel, median over the sweep", "peak_source": "of " + which,
+            "min_frac": fr[0], "max_frac": fr[-1]}
+    return total_ms, launches, roof, clocks, {"sweep": rows, "units": total_units,
+                                               "l2": "n >= 8 rows of 16.8 MB per array exceed L2; smaller n partly L2-resident"}
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -384,11 +435,13 @@ def main():
     import paper_2306_00256_b200 as ceca
     ceca.library()
 
-    fn = {"step": bench_step, "consensus": bench_consensus, "logreg": bench_logreg}[wl["kind"]]
+    fn = {"step": bench_step, "consensus": bench_consensus, "logreg": bench_logreg, "sweep": bench_sweep}[wl["kind"]]
     total_ms, launches, roof, clocks, extra = fn(args, wl, device, dist)
     total_ms = max_over_ranks(total_ms, dist, device)
     units_per_step = wl["n"] * wl["d"]
     value = world * units_per_step * args.steps / (total_ms * 1e-3)
+    if wl["kind"] == "sweep":
+        value = world * extra.pop("units") / (total_ms * 1e-3)
 
     e2e = None
     if wl["kind"] == "step" and not args.no_e2e:

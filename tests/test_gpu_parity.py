@@ -82,6 +82,45 @@ def test_step_matches_oracle_every_round(n, d):
             assert torch.equal(X, Xo) and torch.equal(Y, Yo)
 
 
+def test_step_every_n_from_2_to_130():
+    """Every agent count of the n sweep (and the paper's n = 130), every round, both variants."""
+    d, gamma = 260, 0.1
+    for n in list(range(2, 131)):
+        x, y, g = synth.step_inputs(n, d, seed=n, x_std=1.0, g_std=1.0, same_xy=False)
+        X0, Y0, G = x.to(DEV), y.to(DEV), g.to(DEV)
+        xn, yn, gn = _np(x), _np(y), _np(g)
+        tol = STEP_TOL * _scale(gamma, (x, 1), (y, 1), (g, gamma))
+        for variant in _variants(n):
+            for k in range(_tau(n)):
+                Xo, Yo = torch.empty_like(X0), torch.empty_like(Y0)
+                ceca.ceca_gossip_sgd_step(X0, Y0, G, gamma, variant, k, X_out=Xo, Y_out=Yo)
+                want_x, want_y = oracle.step(xn, yn, gn, np.float32(gamma), variant, k)
+                assert np.abs(_np(Xo) - want_x).max() <= tol, (n, variant, k)
+                assert np.abs(_np(Yo) - want_y).max() <= tol, (n, variant, k)
+
+
+@pytest.mark.parametrize("n,variant", [(130, ceca.CECA_1P), (130, ceca.CECA_2P), (1026, ceca.CECA_1P), (1026, ceca.CECA_2P)])
+def test_consensus_at_the_papers_network_sizes(n, variant):
+    """n = 130 and n = 1026 (Sec. 5, "close to a power of two"): per-round kernel, tau rounds, random x and y;
+    the residue sum_i ||x_i - mean|| drops to rounding level exactly at round tau, not before."""
+    d = 515
+    x = synth.consensus_inputs(n, d, seed=n, offset_rows=False)
+    y = synth.consensus_inputs(n, d, seed=n + 1, offset_rows=False)
+    tau = _tau(n)
+    mean = x.double().mean(0)
+    X, Y = x.to(DEV), y.to(DEV)
+    for k in range(tau):
+        ceca.ceca_consensus_rounds(X, Y, variant, k, 1, 0)
+        residue = float((X.double().cpu() - mean).norm(dim=1).sum())
+        if k < tau - 1:
+            assert residue > 1e-2 * n
+        else:
+            assert residue < 1e-4 * n
+    want_x, want_y = oracle.consensus(_np(x), _np(y), variant, 0, tau)
+    tol = STEP_TOL * tau * _scale(0, (x, 1), (y, 1))
+    assert np.abs(_np(X) - want_x).max() <= tol and np.abs(_np(Y) - want_y).max() <= tol
+
+
 @pytest.mark.parametrize("n,d,ld,offset", [(6, 37, 40, 0), (6, 37, 41, 0), (24, 1000, 1024, 4), (24, 1000, 1024, 1),
                                            (97, 513, 517, 3), (100, 4096, 4100, 0)])
 def test_step_padded_rows_and_unaligned_bases(n, d, ld, offset):
