@@ -188,7 +188,8 @@ def bench_step(args, wl, device, dist):
     import synthetic_inputs as synth
 
     n, d, variant, gamma = wl["n"], wl["d"], wl["variant"], wl["gamma"]
-    X, Y, G = synth.step_inputs(n, d, seed=0, x_std=0.01, g_std=0.01, device=device)
+    ld = synth.padded_ld(d)  # rows 128-byte aligned: a warp's 512-byte access then covers exactly four lines
+    X, Y, G = synth.step_inputs(n, d, seed=0, x_std=0.01, g_std=0.01, device=device, ld=ld)
     stream = torch.cuda.current_stream()
     tau = ceca.ceca_schedule(n, variant, 0, peers=False)[0].tau
     k = 0
@@ -232,7 +233,8 @@ def bench_step(args, wl, device, dist):
                                 if any((k_first + s) % tau == r for s in range(args.steps)) else None for r in range(tau)]}
     del X, Y, G
     torch.cuda.empty_cache()
-    return total_ms, launches, roof, clocks, {"tau": tau, "in_place": True, "l2": "inputs (3 x n x d fp32) far larger than L2"}
+    return total_ms, launches, roof, clocks, {"tau": tau, "in_place": True, "ld": ld,
+                                               "l2": "inputs (3 x n x d fp32) far larger than L2"}
 
 
 def bench_step_e2e(args, wl, device):

@@ -3,7 +3,8 @@
  *
  * n simulated agents are the rows of dense row-major fp32 matrices X (the models x_i),
  * Y (the auxiliary models y_i) and G (the stochastic gradients e_i), each n x d with a
- * leading dimension ld >= d counted in elements.  One call applies one iteration of
+ * leading dimension ld >= d counted in elements (for full bandwidth make ld a multiple of 32, so
+ * that every row starts on a 128-byte line: with rows of 25.6M floats this is worth ~4 %).  One call applies one iteration of
  * DSGD-CECA (Algorithm 1), or several CECA consensus rounds (Algorithm 2), to all agents.
  *
  * Conventions shared by every entry point

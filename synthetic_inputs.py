@@ -16,9 +16,20 @@ def _gen(seed, device):
     return g
 
 
-def _randn_rows(n, d, gen, device, mean=0.0, std=1.0, out=None):
+def padded_ld(d, multiple=32):
+    """Smallest leading dimension >= d that keeps every row 128-byte aligned (32 floats)."""
+    return (d + multiple - 1) // multiple * multiple
+
+
+def empty_rows(n, d, device, ld=None):
+    """An [n, d] fp32 view whose rows are ld >= d elements apart (ld = d when not given)."""
+    ld = d if ld is None else ld
+    return torch.empty((n, ld), dtype=torch.float32, device=device)[:, :d]
+
+
+def _randn_rows(n, d, gen, device, mean=0.0, std=1.0, out=None, ld=None):
     """Row by row so that a 10 GB matrix never needs a second 10 GB temporary."""
-    x = out if out is not None else torch.empty((n, d), dtype=torch.float32, device=device)
+    x = out if out is not None else empty_rows(n, d, device, ld)
     for i in range(n):
         x[i].normal_(mean=mean, std=std, generator=gen)
     return x
@@ -34,13 +45,18 @@ def consensus_inputs(n, d, seed=1, offset_rows=True, device="cpu"):
     return x
 
 
-def step_inputs(n, d, seed=0, x_std=0.01, g_std=0.01, device="cpu", same_xy=True):
+def step_inputs(n, d, seed=0, x_std=0.01, g_std=0.01, device="cpu", same_xy=True, ld=None):
     """Flat parameter vectors of a CNN's size: X0 iid N(0, x_std^2) per element, Y0 = X0
-    (or an independent draw when ``same_xy`` is false), G iid N(0, g_std^2)."""
+    (or an independent draw when ``same_xy`` is false), G iid N(0, g_std^2).  With ``ld`` the
+    three matrices are [n, d] views of [n, ld] buffers (padded rows)."""
     gen = _gen(seed, device)
-    x = _randn_rows(n, d, gen, device, std=x_std)
-    y = x.clone() if same_xy else _randn_rows(n, d, gen, device, std=x_std)
-    g = _randn_rows(n, d, gen, device, std=g_std)
+    x = _randn_rows(n, d, gen, device, std=x_std, ld=ld)
+    if same_xy:
+        y = empty_rows(n, d, device, ld)
+        y.copy_(x)
+    else:
+        y = _randn_rows(n, d, gen, device, std=x_std, ld=ld)
+    g = _randn_rows(n, d, gen, device, std=g_std, ld=ld)
     return x, y, g
 
 

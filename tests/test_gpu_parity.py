@@ -435,7 +435,9 @@ def test_full_size_step_on_column_windows(n, d, variant, iters):
     """Flat CNN-sized parameter vectors (ResNet-18 / ResNet-50 sized), in place, the launch shape the
     benchmark times; windows include the first and the last (ragged) columns."""
     _need_free(int(3.3 * n * d * 4))
-    X, Y, G = synth.step_inputs(n, d, seed=4, x_std=0.01, g_std=0.01, device=DEV)
+    ld = synth.padded_ld(d)   # the benchmark's layout: rows padded to a multiple of 128 bytes
+    X, Y, G = synth.step_inputs(n, d, seed=4, x_std=0.01, g_std=0.01, device=DEV, ld=ld)
+    assert X.stride(0) == ld and ld % 32 == 0 and d % 32 != 0
     gamma = 0.1
     wins = _windows(d, 4099, 4, seed=n)
     ref = [(_np(X[:, lo:hi]).astype(np.float64), _np(Y[:, lo:hi]).astype(np.float64)) for lo, hi in wins]
