@@ -42,6 +42,9 @@ WORKLOADS = {
     "step_small": dict(kind="step", n=100, d=2_097_152, variant=2, gamma=0.1),
     "consensus_fused": dict(kind="consensus", n=97, d=1 << 20, variant=2, fused=1),
     "consensus_rounds": dict(kind="consensus", n=97, d=1 << 20, variant=2, fused=0),
+    # the paper's larger network size (Sec. 5): 8-column tiles, eleven rounds
+    "consensus_fused_1026": dict(kind="consensus", n=1026, d=1 << 18, variant=2, fused=1),
+    "consensus_rounds_1026": dict(kind="consensus", n=1026, d=1 << 18, variant=2, fused=0),
     "logreg_grad": dict(kind="logreg", n=63, m=2000, d=4096, variant=2, gamma=0.01),
     # n = 2..128 at d = 4,194,304, both variants where defined: kernel and schedule scaling with n
     "n_sweep": dict(kind="sweep", n=128, d=4_194_304, variant=2, gamma=0.1),
@@ -317,7 +320,7 @@ def bench_consensus(args, wl, device, dist):
             "peak_source": "of " + which}
     launches = args.steps * (1 if fused else tau)
     return total_ms, launches, roof, clocks, {"tau": tau, "rounds_per_step": tau,
-                                               "l2": "X is 407 MB, larger than L2; outputs go to separate buffers"}
+                                               "l2": "X is %d MB, larger than L2; outputs go to separate buffers" % (n * d * 4 // 1000000)}
 
 
 def bench_logreg(args, wl, device, dist):

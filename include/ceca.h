@@ -40,7 +40,7 @@ typedef enum {
   CECA_ERR_INVALID_ARG = 1, /* NULL where data is needed, n < 1, d < 1, ld < d, k < 0, ...       */
   CECA_ERR_ODD_N_1P = 2,    /* CECA-1P is defined for even n only (Sec. 3.2)                     */
   CECA_ERR_ALIGNMENT = 3,   /* the fused consensus kernel needs 16-byte aligned rows             */
-  CECA_ERR_UNSUPPORTED = 4, /* e.g. in-place aliasing of only one of X/Y, fused path with n > 256 */
+  CECA_ERR_UNSUPPORTED = 4, /* e.g. crossed aliasing of X/Y buffers, fused path with n > 2048      */
   CECA_ERR_WORKSPACE = 5,   /* workspace NULL or smaller than ceca_workspace_bytes says          */
   CECA_ERR_CUDA = 6,        /* a CUDA runtime / driver call failed (launch, copy, map encode)    */
   CECA_ERR_STATIC_SCRATCH = 7 /* dsgd_logreg_grad_static: the problem needs more scratch than the
@@ -104,7 +104,8 @@ ceca_status_t ceca_gossip_sgd_step(const float *X, const float *Y, const float *
  *              ld and alignment.  Y_out == NULL is allowed when workspace holds n*ld floats.
  *   fused = 1: a single launch.  A column tile of all n rows is brought into shared memory by
  *              TMA (cp.async.bulk.tensor), every round runs on chip, and the tile is written
- *              back once.  Needs n <= 256, X / X_out (and Y / Y_out when used) 16-byte aligned
+ *              back once.  Needs n <= 2048 (32-column tiles up to n = 256, 8-column tiles above),
+ *              X / X_out (and Y / Y_out when used) 16-byte aligned
  *              with ld*4 a multiple of 16 (else CECA_ERR_ALIGNMENT), ld < 2^32, rounds <= 64,
  *              and a workspace of ceca_workspace_bytes(CECA_WS_CONSENSUS_FUSED, ...) bytes
  *              whose first int32 is a status word: it is left unchanged when the launch

@@ -10,7 +10,9 @@
 //   packed two-wide fp32 FMAs; eight columns per thread keep the index arithmetic per element
 //   small).  The finished tiles go back with one TMA tensor store each.  HBM sees X once in and
 //   X (and Y) once out, instead of once per round.  Several CTAs per SM overlap each other's
-//   load, compute and store phases.
+//   load, compute and store phases.  Tiles are 32 columns wide for n <= 256 (one TMA box); for
+//   256 < n <= 2048 they are 8 columns wide and made of several boxes, so that all rows still fit
+//   in shared memory.
 #include <cuda.h>
 #include <cuda_runtime.h>
 
@@ -28,11 +30,11 @@ cudaError_t enqueue_step(const Plan &plan, const float *X, const float *Y, const
 ceca_status_t check_matrix_args(const void *X, const void *X_out, int32_t n, int64_t d, int64_t ld);
 
 constexpr int kMaxFusedRounds = 64;
-constexpr int kMaxFusedRows = 256;   // one TMA box holds at most 256 rows
-constexpr int kTileCols = 32;        // W: columns per CTA tile (128-byte row segments)
+constexpr int kMaxBoxRows = 256;     // one TMA box holds at most 256 rows; taller tiles take several boxes
+constexpr int kWideTileCols = 32;    // W for n <= 256: 128-byte row segments
+constexpr int kNarrowTileCols = 8;   // W for 256 < n <= 2048: 32-byte row segments, so that all rows still fit
+constexpr int kMaxFusedRows = 2048;
 constexpr int kFusedThreads = 256;
-constexpr int kColGroups = 4;                             // a thread owns 2 x 4 columns: groups cg and cg + 4
-constexpr int kRowGroups = kFusedThreads / kColGroups;    // Q = 64: rows are dealt round-robin to Q threads
 constexpr uint32_t kWaitPolls = 1u << 22;  // bounded mbarrier wait (each poll sleeps ~100 ns)
 
 struct FusedRound {
@@ -43,6 +45,7 @@ struct FusedRound {
 
 struct FusedArgs {
   int32_t n, rounds, one_port, has_y_in, has_y_out;
+  int32_t boxes, box_rows;  // the tile is `boxes` TMA boxes of `box_rows` rows (boxes * box_rows >= n)
   int32_t *status;
   FusedRound rd[kMaxFusedRounds];
 };
@@ -98,29 +101,36 @@ __device__ __forceinline__ float4 mix4(float w_own, float4 own, float w_recv, fl
   return make_float4(lo.x, lo.y, hi.x, hi.y);
 }
 
-// R = rows per thread (compile time), so n <= R * kRowGroups.
+// R = rows per thread, W = tile width in columns (both compile time).
 //
-// Thread layout: cg = tid % 4, q = tid / 4.  A thread owns rows q, q + 64, ... and, in each, the two
-// float4 column groups cg and cg + 4 (columns 4 cg .. 4 cg + 3 and 16 + 4 cg .. 16 + 4 cg + 3).
-// It touches them in the order (cg, cg + 4) when q is even and (cg + 4, cg) when q is odd, so the
-// eight threads that share a 128-bit shared-memory transaction (two adjacent row groups) cover
-// all 32 banks: rows are 128 bytes apart and would otherwise collide.
-template <int R>
+// Thread layout: a thread owns eight columns (two float4) of each of its rows.  With COLG = W / 8
+// column groups per row and Q = 256 / COLG row groups: cg = tid % COLG, q = tid / COLG, rows
+// q, q + Q, ..., so n <= R * Q.  The two float4 of a row sit at column groups cg and cg + COLG; a
+// thread touches them in that order or swapped, depending on a bit of q chosen such that the eight
+// threads sharing a 128-bit shared-memory transaction cover all 32 banks:
+//   W = 32 (rows 128 bytes apart): two adjacent row groups share a transaction -> swap on q & 1;
+//   W = 8  (rows  32 bytes apart): eight adjacent rows share it              -> swap on (q >> 2) & 1.
+template <int R, int W>
 __global__ void __launch_bounds__(kFusedThreads)
 consensus_fused_kernel(const __grid_constant__ CUtensorMap map_x_in, const __grid_constant__ CUtensorMap map_y_in,
                        const __grid_constant__ CUtensorMap map_x_out,
                        const __grid_constant__ CUtensorMap map_y_out, const __grid_constant__ FusedArgs p) {
+  constexpr int kTileCols = W;
+  constexpr int kColGroups = W / 8;
+  constexpr int kRowGroups = kFusedThreads / kColGroups;
   extern __shared__ __align__(128) unsigned char smem_raw[];
   const int n = p.n;
   float *tile_a = reinterpret_cast<float *>(smem_raw);            // [n][W]  X tile, then exchange buffer
-  float *tile_b = tile_a + (size_t)n * kTileCols;                 // [n][W]  Y tile, then exchange buffer
+  const int tile_rows = p.boxes * p.box_rows;                     // >= n; the surplus rows are never used
+  float *tile_b = tile_a + (size_t)tile_rows * kTileCols;         // [n][W]  Y tile, then exchange buffer
   __shared__ __align__(8) uint64_t bar;
 
   const int cg = threadIdx.x % kColGroups;
   const int q = threadIdx.x / kColGroups;
-  const int c0 = 4 * (cg + 4 * (q & 1));        // columns of the float4 touched first
-  const int c1 = 4 * (cg + 4 * ((q & 1) ^ 1));  // ... and second
-  const int32_t col0 = (int32_t)blockIdx.x * kTileCols;  // multiple of 32 floats: 16-byte aligned
+  const int swap = (W == 32) ? (q & 1) : ((q >> 2) & 1);
+  const int c0 = 4 * (cg + kColGroups * swap);        // columns of the float4 touched first
+  const int c1 = 4 * (cg + kColGroups * (swap ^ 1));  // ... and second
+  const int32_t col0 = (int32_t)blockIdx.x * kTileCols;  // a multiple of 8 floats: 16-byte aligned
 
   if (threadIdx.x == 0) {
     mbar_init(&bar, 1);
@@ -128,10 +138,13 @@ consensus_fused_kernel(const __grid_constant__ CUtensorMap map_x_in, const __gri
   }
   __syncthreads();
   if (threadIdx.x == 0) {
-    const uint32_t tile_bytes = (uint32_t)n * kTileCols * sizeof(float);
+    const uint32_t tile_bytes = (uint32_t)tile_rows * kTileCols * sizeof(float);  // boxes count in full
     mbar_expect_tx(&bar, p.has_y_in ? 2 * tile_bytes : tile_bytes);
-    tma_load_2d(tile_a, &map_x_in, col0, 0, &bar);
-    if (p.has_y_in) tma_load_2d(tile_b, &map_y_in, col0, 0, &bar);
+    for (int b = 0; b < p.boxes; ++b) {  // rows past n are out of range for the tensor map: zero fill
+      const int row0 = b * p.box_rows;
+      tma_load_2d(tile_a + (size_t)row0 * kTileCols, &map_x_in, col0, row0, &bar);
+      if (p.has_y_in) tma_load_2d(tile_b + (size_t)row0 * kTileCols, &map_y_in, col0, row0, &bar);
+    }
   }
   const bool landed = mbar_wait_bounded(&bar, 0, kWaitPolls);
   if (!__syncthreads_and(landed)) {  // one decision for the whole CTA
@@ -223,8 +236,11 @@ consensus_fused_kernel(const __grid_constant__ CUtensorMap map_x_in, const __gri
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic writes -> visible to TMA
   __syncthreads();
   if (threadIdx.x == 0) {
-    tma_store_2d(&map_x_out, col0, 0, tile_a);
-    if (p.has_y_out) tma_store_2d(&map_y_out, col0, 0, tile_b);
+    for (int b = 0; b < p.boxes; ++b) {  // the tensor map clips rows >= n and columns >= d
+      const int row0 = b * p.box_rows;
+      tma_store_2d(&map_x_out, col0, row0, tile_a + (size_t)row0 * kTileCols);
+      if (p.has_y_out) tma_store_2d(&map_y_out, col0, row0, tile_b + (size_t)row0 * kTileCols);
+    }
     asm volatile("cp.async.bulk.commit_group;" ::: "memory");
     asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");  // smem must outlive the reads
   }
@@ -248,31 +264,32 @@ static EncodeTiledFn encode_tiled_fn() {
   return fn;
 }
 
-// An n x d fp32 matrix with row pitch ld, boxed as n rows x kTileCols columns.
-static bool make_map(CUtensorMap *map, const float *base, int32_t n, int64_t d, int64_t ld) {
+// An n x d fp32 matrix with row pitch ld, boxed as box_rows rows x tile_cols columns.
+static bool make_map(CUtensorMap *map, const float *base, int32_t n, int64_t d, int64_t ld, int tile_cols,
+                     int box_rows) {
   EncodeTiledFn enc = encode_tiled_fn();
   if (!enc) return false;
   const cuuint64_t dims[2] = {(cuuint64_t)d, (cuuint64_t)n};
   const cuuint64_t strides[1] = {(cuuint64_t)ld * sizeof(float)};
-  const cuuint32_t box[2] = {(cuuint32_t)kTileCols, (cuuint32_t)n};
+  const cuuint32_t box[2] = {(cuuint32_t)tile_cols, (cuuint32_t)box_rows};
   const cuuint32_t elem[2] = {1, 1};
   return enc(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float *>(base), dims, strides, box, elem,
              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int R>
+template <int R, int W>
 static cudaError_t launch_fused(const CUtensorMap &mxi, const CUtensorMap &myi, const CUtensorMap &mxo,
                                 const CUtensorMap &myo, const FusedArgs &args, int64_t d, cudaStream_t stream) {
-  const size_t smem = 2 * (size_t)args.n * kTileCols * sizeof(float);
-  cudaError_t e = cudaFuncSetAttribute(consensus_fused_kernel<R>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  const size_t smem = 2 * (size_t)args.boxes * args.box_rows * W * sizeof(float);
+  cudaError_t e = cudaFuncSetAttribute(consensus_fused_kernel<R, W>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        (int)smem);
   if (e != cudaSuccess) return e;
-  e = cudaFuncSetAttribute(consensus_fused_kernel<R>, cudaFuncAttributePreferredSharedMemoryCarveout,
+  e = cudaFuncSetAttribute(consensus_fused_kernel<R, W>, cudaFuncAttributePreferredSharedMemoryCarveout,
                            cudaSharedmemCarveoutMaxShared);
   if (e != cudaSuccess) return e;
-  const int64_t tiles = (d + kTileCols - 1) / kTileCols;
-  consensus_fused_kernel<R><<<(unsigned)tiles, kFusedThreads, smem, stream>>>(mxi, myi, mxo, myo, args);
+  const int64_t tiles = (d + W - 1) / W;
+  consensus_fused_kernel<R, W><<<(unsigned)tiles, kFusedThreads, smem, stream>>>(mxi, myi, mxo, myo, args);
   return cudaGetLastError();
 }
 
@@ -306,17 +323,34 @@ static ceca_status_t consensus_fused(const float *X, const float *Y, float *Xo, 
       (Yo && !aligned16(Yo)))
     return CECA_ERR_ALIGNMENT;
 
+  // tile geometry: all n rows, 32 columns wide while one TMA box (256 rows) holds them, else 8
+  const int tile_cols = n <= kMaxBoxRows ? kWideTileCols : kNarrowTileCols;
+  args.boxes = (n + kMaxBoxRows - 1) / kMaxBoxRows;
+  args.box_rows = (n + args.boxes - 1) / args.boxes;
+  if (tile_cols == kNarrowTileCols)  // every box must start on a 128-byte boundary of shared memory
+    args.box_rows = (args.box_rows + 3) / 4 * 4;
   CUtensorMap mxi, myi, mxo, myo;
-  if (!make_map(&mxi, X, n, d, ld) || !make_map(&mxo, Xo, n, d, ld)) return CECA_ERR_CUDA;
-  if (!make_map(&myi, args.has_y_in ? Y : X, n, d, ld)) return CECA_ERR_CUDA;
-  if (!make_map(&myo, Yo ? Yo : Xo, n, d, ld)) return CECA_ERR_CUDA;
+  if (!make_map(&mxi, X, n, d, ld, tile_cols, args.box_rows) || !make_map(&mxo, Xo, n, d, ld, tile_cols, args.box_rows))
+    return CECA_ERR_CUDA;
+  if (!make_map(&myi, args.has_y_in ? Y : X, n, d, ld, tile_cols, args.box_rows)) return CECA_ERR_CUDA;
+  if (!make_map(&myo, Yo ? Yo : Xo, n, d, ld, tile_cols, args.box_rows)) return CECA_ERR_CUDA;
 
-  const int rows_per_thread = (n + kRowGroups - 1) / kRowGroups;  // n <= 256 -> at most 4
   cudaError_t e;
-  if (rows_per_thread <= 1)      e = launch_fused<1>(mxi, myi, mxo, myo, args, d, stream);
-  else if (rows_per_thread <= 2) e = launch_fused<2>(mxi, myi, mxo, myo, args, d, stream);
-  else if (rows_per_thread <= 3) e = launch_fused<3>(mxi, myi, mxo, myo, args, d, stream);
-  else                           e = launch_fused<4>(mxi, myi, mxo, myo, args, d, stream);
+  if (tile_cols == kWideTileCols) {
+    const int rows_per_thread = (n + 63) / 64;  // 64 row groups; n <= 256 -> at most 4
+    if (rows_per_thread <= 1)      e = launch_fused<1, kWideTileCols>(mxi, myi, mxo, myo, args, d, stream);
+    else if (rows_per_thread <= 2) e = launch_fused<2, kWideTileCols>(mxi, myi, mxo, myo, args, d, stream);
+    else if (rows_per_thread <= 3) e = launch_fused<3, kWideTileCols>(mxi, myi, mxo, myo, args, d, stream);
+    else                           e = launch_fused<4, kWideTileCols>(mxi, myi, mxo, myo, args, d, stream);
+  } else {
+    const int rows_per_thread = (n + 255) / 256;  // 256 row groups; n <= 2048 -> at most 8
+    if (rows_per_thread <= 2)      e = launch_fused<2, kNarrowTileCols>(mxi, myi, mxo, myo, args, d, stream);
+    else if (rows_per_thread <= 3) e = launch_fused<3, kNarrowTileCols>(mxi, myi, mxo, myo, args, d, stream);
+    else if (rows_per_thread <= 4) e = launch_fused<4, kNarrowTileCols>(mxi, myi, mxo, myo, args, d, stream);
+    else if (rows_per_thread <= 5) e = launch_fused<5, kNarrowTileCols>(mxi, myi, mxo, myo, args, d, stream);
+    else if (rows_per_thread <= 6) e = launch_fused<6, kNarrowTileCols>(mxi, myi, mxo, myo, args, d, stream);
+    else                           e = launch_fused<8, kNarrowTileCols>(mxi, myi, mxo, myo, args, d, stream);
+  }
   return e == cudaSuccess ? CECA_OK : CECA_ERR_CUDA;
 }
 

@@ -227,6 +227,31 @@ def test_consensus_matches_oracle_and_reaches_the_mean(fused, n, d):
             assert torch.equal(X, Xo) and torch.equal(Y, Yo)
 
 
+@pytest.mark.parametrize("n", [257, 300, 514, 1026, 1300, 2047, 2048])
+@pytest.mark.parametrize("d", [8, 1000, 4100])
+def test_fused_consensus_above_256_agents(n, d):
+    """Narrow (8-column) tiles made of several TMA boxes: tau rounds, extra rounds, unaligned starts."""
+    x = synth.consensus_inputs(n, d, seed=n + d)
+    y0 = synth.consensus_inputs(n, d, seed=n + d + 1, offset_rows=False)
+    tau = _tau(n)
+    for variant in _variants(n):
+        for k0, rounds in [(0, tau), (3, tau + 2), (tau, 1)]:
+            X, Y = x.to(DEV), y0.to(DEV)
+            Xo, Yo = torch.full_like(X, float("nan")), torch.full_like(Y, float("nan"))
+            ws = _fused_ws()
+            ceca.ceca_consensus_rounds(X, Y, variant, k0, rounds, 1, X_out=Xo, Y_out=Yo, workspace=ws)
+            assert ceca.ceca_read_status(ws) == 0
+            want_x, want_y = oracle.consensus(_np(x), _np(y0), variant, k0, rounds)
+            tol = STEP_TOL * rounds * _scale(0, (x, 1), (y0, 1))
+            assert np.abs(_np(Xo) - want_x).max() <= tol, (n, d, variant, k0, rounds)
+            assert np.abs(_np(Yo) - want_y).max() <= tol, (n, d, variant, k0, rounds)
+            if k0 == 0:
+                xd = Xo.double()
+                assert float((xd - x.double().mean(0).to(DEV)).norm() / xd.norm()) <= 1e-5
+            ceca.ceca_consensus_rounds(X, Y, variant, k0, rounds, 1, workspace=ws)   # in place: same bits
+            assert torch.equal(X, Xo) and torch.equal(Y, Yo)
+
+
 @pytest.mark.parametrize("fused", [0, 1])
 def test_consensus_optional_y(fused):
     n, d = 97, 1000
