@@ -40,6 +40,8 @@ WORKLOADS = {
     # smaller cases of the same kernels, for profiler captures and quick looks
     "resnet18_step": dict(kind="step", n=24, d=11_689_512, variant=1, gamma=0.1),
     "step_small": dict(kind="step", n=100, d=2_097_152, variant=2, gamma=0.1),
+    # n a power of two: the X-only update (12 B per agent-parameter; CECA-2P = one-peer exponential graph)
+    "pow2_xonly_step": dict(kind="step", n=128, d=8_388_608, variant=2, gamma=0.1, x_only=True),
     "consensus_fused": dict(kind="consensus", n=97, d=1 << 20, variant=2, fused=1),
     "consensus_rounds": dict(kind="consensus", n=97, d=1 << 20, variant=2, fused=0),
     # the paper's larger network size (Sec. 5): 8-column tiles, eleven rounds
@@ -195,6 +197,9 @@ def bench_step(args, wl, device, dist):
     X, Y, G = synth.step_inputs(n, d, seed=0, x_std=0.01, g_std=0.01, device=device, ld=ld)
     stream = torch.cuda.current_stream()
     tau = ceca.ceca_schedule(n, variant, 0, peers=False)[0].tau
+    x_only = bool(wl.get("x_only"))
+    if x_only:
+        Y = None
     k = 0
     for _ in range(args.warmup):
         ceca.ceca_gossip_sgd_step(X, Y, G, gamma, variant, k)
@@ -219,17 +224,17 @@ def bench_step(args, wl, device, dist):
     per_launch = [events[s].elapsed_time(events[s + 1]) for s in range(args.steps)]
     # dominant kernel: the launches that read Y (every round but r = 0), 20 B per agent-parameter
     dominant = [per_launch[s] for s in range(args.steps)
-                if ceca.ceca_schedule(n, variant, k_first + s, peers=False)[0].b_num != 0
+                if x_only or ceca.ceca_schedule(n, variant, k_first + s, peers=False)[0].b_num != 0
                 or ceca.ceca_schedule(n, variant, k_first + s, peers=False)[0].payload == 1]
     launches = args.steps * (1 if d % 4 == 0 else 2)
     roof = None
     if dominant:
         avg_ms = sum(dominant) / len(dominant)
         peak, which = measured_peak()
-        achieved = algorithmic_bytes_step(n, d, True) / (avg_ms * 1e-3) / 1e9
+        achieved = (12 * n * d if x_only else algorithmic_bytes_step(n, d, True)) / (avg_ms * 1e-3) / 1e9
         roof = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                 "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH.get(args.workload),
-                "kernel": "step_walk_kernel<float4, gradient, reads Y>", "peak_source": "of " + which,
+                "kernel": "step_walk_kernel<float4, gradient, %s>" % ("X only" if x_only else "reads Y"), "peak_source": "of " + which,
                 "avg_launch_ms": avg_ms, "launches_timed": len(dominant),
                 "frac_of_nominal_8TBs": achieved / 8000.0,
                 "ms_by_round": [round(statistics.mean(per_launch[s] for s in range(args.steps) if (k_first + s) % tau == r), 4)
@@ -449,7 +454,7 @@ def main():
         value = world * extra.pop("units") / (total_ms * 1e-3)
 
     e2e = None
-    if wl["kind"] == "step" and not args.no_e2e:
+    if wl["kind"] == "step" and not args.no_e2e and not wl.get("x_only"):
         e2e = bench_step_e2e(args, wl, device)
         if dist is not None:
             ms = max_over_ranks(e2e["ms_per_step"], dist, device)

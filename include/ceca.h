@@ -87,6 +87,10 @@ ceca_status_t ceca_schedule(int32_t n, ceca_variant_t variant, int64_t k, ceca_r
  * Y_out == Y (in place: every element is read and then written by the same thread).  A crossed
  * alias (X_out == Y, Y_out == X, an output equal to G, X_out == Y_out) is CECA_ERR_UNSUPPORTED;
  * partially overlapping buffers are not detected and give undefined results.
+ * X-only form: when n is a power of two every delta_r is 1 (Sec. 3.1), every message is built from
+ * x, and X never depends on Y (CECA-2P is then the one-peer exponential graph).  Passing Y == NULL
+ * and Y_out == NULL runs just the x update: 12 bytes per agent-parameter instead of 20.  For any
+ * other n this combination is CECA_ERR_INVALID_ARG.
  * fp32 arithmetic; a, b and 1-a, 1-b are formed in fp64 on the host and rounded once.
  */
 ceca_status_t ceca_gossip_sgd_step(const float *X, const float *Y, const float *G, float *X_out,

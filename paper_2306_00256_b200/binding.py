@@ -120,13 +120,12 @@ def ceca_schedule(n, variant, k, peers=True):
 
 
 def ceca_gossip_sgd_step(X, Y, G, gamma, variant, k, X_out=None, Y_out=None, stream=None):
-    """One DSGD-CECA iteration on device tensors.  Outputs default to in place.  Returns (X_out, Y_out)."""
+    """One DSGD-CECA iteration on device tensors.  Outputs default to in place.  Returns (X_out, Y_out).
+    Y = Y_out = None asks for the X-only update (n a power of two)."""
     n, d, ld = _matrix(X, "X")
     X_out = X if X_out is None else X_out
-    if Y_out is None:
-        if Y is None:
-            raise ValueError("Y_out is needed when Y is None")
-        Y_out = Y
+    if Y_out is None and Y is not None:
+        Y_out = Y   # (Y and Y_out both None: the X-only update, legal for n a power of two)
     for t, name in ((Y, "Y"), (G, "G"), (X_out, "X_out"), (Y_out, "Y_out")):
         if t is not None and _matrix(t, name, n) != (n, d, ld):
             raise ValueError("%s must have the shape and row stride of X" % name)

@@ -68,8 +68,11 @@ struct RowRegs {
 // RIF = rows whose loads are issued before any of them is consumed (memory-level parallelism per
 // thread); MINB = CTAs per SM the register allocation must allow (parallelism across threads).
 // Long cycles want a deep RIF, cycles of two rows have only two rows to load and want occupancy.
-template <typename V, bool HAS_G, bool USE_Y, int RIF, int MINB>
+// YMODE: 1 = Y is read and written; 0 = Y has zero weight this round, it is only written;
+//        2 = X only (n a power of two: every round builds its message from x, so X never depends on Y).
+template <typename V, bool HAS_G, int YMODE, int RIF, int MINB>
 __global__ void __launch_bounds__(kThreads, MINB) step_walk_kernel(const StepArgs p) {
+  constexpr bool USE_Y = (YMODE == 1);
   constexpr int VW = sizeof(V) / sizeof(float);
   const int64_t colv = (int64_t)blockIdx.x * kThreads + threadIdx.x;
   if (colv >= p.ncolv) return;
@@ -107,7 +110,7 @@ __global__ void __launch_bounds__(kThreads, MINB) step_walk_kernel(const StepArg
           V own_x, own_y, u;
           batch[j].own_terms(p, own_x, own_y, u);
           vstore<V>(p.Xo + offs[j], vfma(p.a, own_x, vmul(p.one_minus_a, u_prev)));
-          vstore<V>(p.Yo + offs[j], vfma(p.b, own_y, vmul(p.one_minus_b, u_prev)));
+          if (YMODE != 2) vstore<V>(p.Yo + offs[j], vfma(p.b, own_y, vmul(p.one_minus_b, u_prev)));
           u_prev = u;
         }
       }
@@ -115,21 +118,23 @@ __global__ void __launch_bounds__(kThreads, MINB) step_walk_kernel(const StepArg
     if (!first_done) first.own_terms(p, first_own_x, first_own_y, u_prev);  // cycle of one row
     // close the cycle: the first row receives the message of the last one
     vstore<V>(p.Xo + first_off, vfma(p.a, first_own_x, vmul(p.one_minus_a, u_prev)));
-    vstore<V>(p.Yo + first_off, vfma(p.b, first_own_y, vmul(p.one_minus_b, u_prev)));
+    if (YMODE != 2) vstore<V>(p.Yo + first_off, vfma(p.b, first_own_y, vmul(p.one_minus_b, u_prev)));
   }
 }
 
 template <typename V, int RIF, int MINB>
-static cudaError_t launch_walk_shape(const StepArgs &args, bool has_g, bool use_y, cudaStream_t stream) {
+static cudaError_t launch_walk_shape(const StepArgs &args, bool has_g, int ymode, cudaStream_t stream) {
   const int64_t blocks_x = (args.ncolv + kThreads - 1) / kThreads;
   if (blocks_x > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
   dim3 grid((unsigned)blocks_x, (unsigned)(args.n_cycles < 65535 ? args.n_cycles : 65535));
   if (has_g) {
-    if (use_y) step_walk_kernel<V, true, true, RIF, MINB><<<grid, kThreads, 0, stream>>>(args);
-    else       step_walk_kernel<V, true, false, RIF, MINB><<<grid, kThreads, 0, stream>>>(args);
+    if (ymode == 1)      step_walk_kernel<V, true, 1, RIF, MINB><<<grid, kThreads, 0, stream>>>(args);
+    else if (ymode == 0) step_walk_kernel<V, true, 0, RIF, MINB><<<grid, kThreads, 0, stream>>>(args);
+    else                 step_walk_kernel<V, true, 2, RIF, MINB><<<grid, kThreads, 0, stream>>>(args);
   } else {
-    if (use_y) step_walk_kernel<V, false, true, RIF, MINB><<<grid, kThreads, 0, stream>>>(args);
-    else       step_walk_kernel<V, false, false, RIF, MINB><<<grid, kThreads, 0, stream>>>(args);
+    if (ymode == 1)      step_walk_kernel<V, false, 1, RIF, MINB><<<grid, kThreads, 0, stream>>>(args);
+    else if (ymode == 0) step_walk_kernel<V, false, 0, RIF, MINB><<<grid, kThreads, 0, stream>>>(args);
+    else                 step_walk_kernel<V, false, 2, RIF, MINB><<<grid, kThreads, 0, stream>>>(args);
   }
   return cudaGetLastError();
 }
@@ -138,18 +143,19 @@ static cudaError_t launch_walk_shape(const StepArgs &args, bool has_g, bool use_
 // cycles of two rows (every CECA-1P round, and the 2-port shift n/2) have nothing to pipeline and
 // run fastest with many resident CTAs; long walks want four rows of loads in flight per thread.
 template <typename V>
-static cudaError_t launch_walk(const StepArgs &args, bool has_g, bool use_y, cudaStream_t stream) {
+static cudaError_t launch_walk(const StepArgs &args, bool has_g, int ymode, cudaStream_t stream) {
   if (args.ncolv <= 0) return cudaSuccess;
   if (args.cycle_len <= 2)
-    return use_y ? launch_walk_shape<V, 1, 4>(args, has_g, use_y, stream)
-                 : launch_walk_shape<V, 1, 6>(args, has_g, use_y, stream);
-  if (args.cycle_len <= 4) return launch_walk_shape<V, 2, 4>(args, has_g, use_y, stream);
-  return launch_walk_shape<V, 4, 2>(args, has_g, use_y, stream);
+    return ymode == 1 ? launch_walk_shape<V, 1, 4>(args, has_g, ymode, stream)
+                      : launch_walk_shape<V, 1, 6>(args, has_g, ymode, stream);
+  if (args.cycle_len <= 4) return launch_walk_shape<V, 2, 4>(args, has_g, ymode, stream);
+  return launch_walk_shape<V, 4, 2>(args, has_g, ymode, stream);
 }
 
 static inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
-// Enqueues one iteration.  Arguments are assumed validated.
+// Enqueues one iteration.  Arguments are assumed validated.  Yo == nullptr selects the X-only update
+// (the caller has checked that n is a power of two).
 cudaError_t enqueue_step(const Plan &plan, const float *X, const float *Y, const float *G, float *Xo,
                          float *Yo, int32_t n, int64_t d, int64_t ld, float gamma,
                          cudaStream_t stream) {
@@ -162,22 +168,23 @@ cudaError_t enqueue_step(const Plan &plan, const float *X, const float *Y, const
   a.a = plan.a; a.b = plan.b; a.one_minus_a = plan.one_minus_a; a.one_minus_b = plan.one_minus_b;
   a.gamma = gamma;
   const bool has_g = (G != nullptr);
-  const bool use_y = plan.reads_y;
-  const bool vec_ok = (ld % 4 == 0) && aligned16(X) && aligned16(Xo) && aligned16(Yo) &&
+  const int ymode = !Yo ? 2 : (plan.reads_y ? 1 : 0);
+  const bool use_y = (ymode == 1);
+  const bool vec_ok = (ld % 4 == 0) && aligned16(X) && aligned16(Xo) && (!Yo || aligned16(Yo)) &&
                       (!use_y || aligned16(Y)) && (!has_g || aligned16(G));
   const int64_t d_vec = vec_ok ? (d / 4) * 4 : 0;  // columns covered by 128-bit accesses
   if (d_vec > 0) {
     a.ncolv = d_vec / 4;
-    cudaError_t e = launch_walk<float4>(a, has_g, use_y, stream);
+    cudaError_t e = launch_walk<float4>(a, has_g, ymode, stream);
     if (e != cudaSuccess) return e;
   }
   if (d_vec < d) {  // ragged tail (or everything, when rows are not 16-byte aligned)
     StepArgs t = a;
-    t.X = X + d_vec; t.Xo = Xo + d_vec; t.Yo = Yo + d_vec;
+    t.X = X + d_vec; t.Xo = Xo + d_vec; t.Yo = Yo ? Yo + d_vec : nullptr;
     t.Y = Y ? Y + d_vec : nullptr;
     t.G = G ? G + d_vec : nullptr;
     t.ncolv = d - d_vec;
-    cudaError_t e = launch_walk<float>(t, has_g, use_y, stream);
+    cudaError_t e = launch_walk<float>(t, has_g, ymode, stream);
     if (e != cudaSuccess) return e;
   }
   return cudaSuccess;
@@ -197,13 +204,17 @@ extern "C" ceca_status_t ceca_gossip_sgd_step(const float *X, const float *Y, co
                                               int64_t k, void *stream) {
   ceca_status_t st = ceca::check_matrix_args(X, X_out, n, d, ld);
   if (st != CECA_OK) return st;
-  if (!Y_out) return CECA_ERR_INVALID_ARG;
   ceca::Plan plan;
   st = ceca::make_plan(n, variant, k, &plan);
   if (st != CECA_OK) return st;
-  if (!Y && plan.reads_y) return CECA_ERR_INVALID_ARG;
+  if (!Y_out) {
+    // X-only update: legal exactly when no round ever builds its message from y, i.e. n-1 is all ones
+    if (Y || (n & (n - 1)) != 0) return CECA_ERR_INVALID_ARG;
+  } else if (!Y && plan.reads_y) {
+    return CECA_ERR_INVALID_ARG;
+  }
   // X_out == X and Y_out == Y are fine (read-then-write by one thread); crossed aliases are not
-  if (X_out == Y_out || (const float *)X_out == Y || (const float *)Y_out == X ||
+  if (X_out == Y_out || (const float *)X_out == Y || (Y_out && (const float *)Y_out == X) ||
       (G && ((const float *)X_out == G || (const float *)Y_out == G)))
     return CECA_ERR_UNSUPPORTED;
   cudaError_t e = ceca::enqueue_step(plan, X, Y, G, X_out, Y_out, n, d, ld, gamma,

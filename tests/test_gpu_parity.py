@@ -161,6 +161,32 @@ def test_step_without_gradient_is_a_ceca_round_and_y_may_be_absent_in_round_zero
             ceca.ceca_gossip_sgd_step(x.to(DEV), None, None, 0.0, variant, 1, X_out=Xo2, Y_out=Yo2)
 
 
+@pytest.mark.parametrize("n", [1, 2, 4, 8, 64, 128])
+@pytest.mark.parametrize("d", [5, 1023, 40004])
+def test_x_only_step_for_power_of_two_agents(n, d):
+    """n = 2^tau: every delta_r is 1, X never depends on Y, and the call without Y must give the oracle's X."""
+    x, y, g = synth.step_inputs(n, d, seed=n + d, x_std=1.0, g_std=1.0, same_xy=False)
+    gamma = 0.1
+    tol = STEP_TOL * _scale(gamma, (x, 1), (g, gamma))
+    for variant in _variants(n):
+        for k in range(_tau(n) + 1):
+            X, G = x.to(DEV), g.to(DEV)
+            Xo = torch.full_like(X, float("nan"))
+            ceca.ceca_gossip_sgd_step(X, None, G, gamma, variant, k, X_out=Xo)
+            want_x, _ = oracle.step(_np(x), _np(y), _np(g), np.float32(gamma), variant, k)
+            assert np.abs(_np(Xo) - want_x).max() <= tol, (n, d, variant, k)
+            # the same bits as the full update's X, and in place
+            Xf, Yf = torch.empty_like(X), torch.empty_like(X)
+            ceca.ceca_gossip_sgd_step(X, y.to(DEV), G, gamma, variant, k, X_out=Xf, Y_out=Yf)
+            assert torch.equal(Xo, Xf)
+            ceca.ceca_gossip_sgd_step(X, None, G, gamma, variant, k)
+            assert torch.equal(X, Xo)
+    if n > 2:   # any other n needs Y
+        bad = torch.zeros(n - 1, d, device=DEV)
+        with pytest.raises(ceca.CecaError):
+            ceca.ceca_gossip_sgd_step(bad, None, None, gamma, ceca.CECA_2P, 0, X_out=torch.empty_like(bad))
+
+
 @pytest.mark.parametrize("n,variant", [(5, ceca.CECA_2P), (6, ceca.CECA_1P), (63, ceca.CECA_2P), (64, ceca.CECA_1P)])
 def test_mean_lemma_and_resume_on_gpu(n, variant):
     """Lemma "relation between averaged variables": with x0 = y0 the mean takes a plain SGD step.
