@@ -48,6 +48,10 @@ WORKLOADS = {
     "consensus_fused_1026": dict(kind="consensus", n=1026, d=1 << 18, variant=2, fused=1),
     "consensus_rounds_1026": dict(kind="consensus", n=1026, d=1 << 18, variant=2, fused=0),
     "logreg_grad": dict(kind="logreg", n=63, m=2000, d=4096, variant=2, gamma=0.01),
+    # whole iterations (gradient kernel + fused step), one CECA cycle captured in a CUDA graph and replayed
+    "logreg_train": dict(kind="train", n=63, m=2000, d=4096, variant=2, gamma=0.01, loss="logistic"),
+    "logreg_train_small": dict(kind="train", n=5, m=100, d=32, variant=2, gamma=0.05, loss="logistic"),
+    "lsq_train": dict(kind="train", n=258, m=50, d=10, variant=1, gamma=0.02, loss="square"),
     # n = 2..128 at d = 4,194,304, both variants where defined: kernel and schedule scaling with n
     "n_sweep": dict(kind="sweep", n=128, d=4_194_304, variant=2, gamma=0.1),
 }
@@ -365,6 +369,69 @@ def bench_logreg(args, wl, device, dist):
     return total_ms, 3 * args.steps, roof, clocks, {"m": m, "l2": "A is 2.06 GB, larger than L2"}
 
 
+def bench_train(args, wl, device, dist):
+    """args.steps CECA cycles of (gradient + fused step): eager launches, then one captured cycle replayed."""
+    import torch
+    import paper_2306_00256_b200 as ceca
+    import synthetic_inputs as synth
+    n, m, d, variant, gamma = wl["n"], wl["m"], wl["d"], wl["variant"], wl["gamma"]
+    if wl["loss"] == "logistic":
+        A, T, _ = synth.logreg_problem(n, m, d, seed=3, flip=0.05, hetero_std=0.5, device=device)
+        grad = lambda X, Y, G, k: ceca.dsgd_logreg_grad(A, T, X, Y, k, variant, G, ws)
+    else:
+        A, T, _ = synth.lsq_problem(n, m, d, seed=0, sigma_s=0.1, device=device)
+        noise = synth.gradient_noise(n, d, 0, sigma_n=5.0, device=device)
+        grad = lambda X, Y, G, k: ceca.dsgd_lsq_grad(A, T, X, Y, k, variant, G, ws, noise=noise)
+    ws = torch.empty(ceca.ceca_workspace_bytes(ceca.WS_LOGREG_GRAD, n, m, d), dtype=torch.uint8, device=device)
+    X = torch.zeros(n, d, device=device); Y = torch.zeros(n, d, device=device); G = torch.empty(n, d, device=device)
+    tau = ceca.ceca_schedule(n, variant, 0, peers=False)[0].tau
+
+    def cycle(k0):
+        for k in range(k0, k0 + tau):
+            grad(X, Y, G, k)
+            ceca.ceca_gossip_sgd_step(X, Y, G, gamma, variant, k)
+
+    stream = torch.cuda.current_stream()
+    e = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+    for c in range(args.warmup):
+        cycle(c * tau)
+    torch.cuda.synchronize()
+    e[0].record(stream)
+    for c in range(args.steps):
+        cycle(c * tau)
+    e[1].record(stream)
+    torch.cuda.synchronize()
+    eager_ms = e[0].elapsed_time(e[1])
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        cycle(0)
+    for _ in range(args.warmup):
+        graph.replay()
+    sampler = ClockSampler(torch.cuda.current_device())
+    sampler.start()
+    stream = torch.cuda.current_stream()
+    torch.cuda.synchronize()
+    e[2].record(stream)
+    for c in range(args.steps):
+        graph.replay()
+    e[3].record(stream)
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    graph_ms = e[2].elapsed_time(e[3])
+    iters = args.steps * tau
+    peak, which = measured_peak()
+    bytes_per_iter = 4 * n * m * d + 8 * n * d + 4 * n * m + (20 * tau - 4) / tau * n * d
+    achieved = bytes_per_iter * iters / (graph_ms * 1e-3) / 1e9
+    roof = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak, "traffic": None,
+            "kernel": "gradient kernels + step_walk_kernel, whole iteration", "peak_source": "of " + which,
+            "note": "launch-latency bound when n*m*d is small"}
+    extra = {"tau": tau, "m": m, "loss": wl["loss"], "iterations_timed": iters, "units": n * d * iters,
+             "eager_us_per_iteration": round(eager_ms / iters * 1e3, 2), "graph_us_per_iteration": round(graph_ms / iters * 1e3, 2),
+             "l2": "A is %.1f MB" % (n * m * d * 4 / 1e6)}
+    launches = iters * (3 if (d % 4 == 0) else 3)
+    return graph_ms, launches, roof, clocks, extra
+
+
 def bench_sweep(args, wl, device, dist):
     """One full CECA cycle (tau fused steps, in place) per n and variant; also the host schedule call."""
     import torch
@@ -445,12 +512,13 @@ def main():
     import paper_2306_00256_b200 as ceca
     ceca.library()
 
-    fn = {"step": bench_step, "consensus": bench_consensus, "logreg": bench_logreg, "sweep": bench_sweep}[wl["kind"]]
+    fn = {"step": bench_step, "consensus": bench_consensus, "logreg": bench_logreg, "sweep": bench_sweep,
+          "train": bench_train}[wl["kind"]]
     total_ms, launches, roof, clocks, extra = fn(args, wl, device, dist)
     total_ms = max_over_ranks(total_ms, dist, device)
     units_per_step = wl["n"] * wl["d"]
     value = world * units_per_step * args.steps / (total_ms * 1e-3)
-    if wl["kind"] == "sweep":
+    if wl["kind"] in ("sweep", "train"):
         value = world * extra.pop("units") / (total_ms * 1e-3)
 
     e2e = None
