@@ -104,20 +104,20 @@ __device__ __forceinline__ float4 mix4(float w_own, float4 own, float w_recv, fl
 // R = rows per thread, W = tile width in columns (both compile time).
 //
 // Thread layout: a thread owns eight columns (two float4) of each of its rows.  With COLG = W / 8
-// column groups per row and Q = 256 / COLG row groups: cg = tid % COLG, q = tid / COLG, rows
+// column groups per row and Q = T / COLG row groups (T threads per CTA): cg = tid % COLG, q = tid / COLG, rows
 // q, q + Q, ..., so n <= R * Q.  The two float4 of a row sit at column groups cg and cg + COLG; a
 // thread touches them in that order or swapped, depending on a bit of q chosen such that the eight
 // threads sharing a 128-bit shared-memory transaction cover all 32 banks:
 //   W = 32 (rows 128 bytes apart): two adjacent row groups share a transaction -> swap on q & 1;
 //   W = 8  (rows  32 bytes apart): eight adjacent rows share it              -> swap on (q >> 2) & 1.
-template <int R, int W>
-__global__ void __launch_bounds__(kFusedThreads)
+template <int R, int W, int T>
+__global__ void __launch_bounds__(T)
 consensus_fused_kernel(const __grid_constant__ CUtensorMap map_x_in, const __grid_constant__ CUtensorMap map_y_in,
                        const __grid_constant__ CUtensorMap map_x_out,
                        const __grid_constant__ CUtensorMap map_y_out, const __grid_constant__ FusedArgs p) {
   constexpr int kTileCols = W;
   constexpr int kColGroups = W / 8;
-  constexpr int kRowGroups = kFusedThreads / kColGroups;
+  constexpr int kRowGroups = T / kColGroups;
   extern __shared__ __align__(128) unsigned char smem_raw[];
   const int n = p.n;
   float *tile_a = reinterpret_cast<float *>(smem_raw);            // [n][W]  X tile, then exchange buffer
@@ -278,18 +278,18 @@ static bool make_map(CUtensorMap *map, const float *base, int32_t n, int64_t d, 
              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int R, int W>
+template <int R, int W, int T>
 static cudaError_t launch_fused(const CUtensorMap &mxi, const CUtensorMap &myi, const CUtensorMap &mxo,
                                 const CUtensorMap &myo, const FusedArgs &args, int64_t d, cudaStream_t stream) {
   const size_t smem = 2 * (size_t)args.boxes * args.box_rows * W * sizeof(float);
-  cudaError_t e = cudaFuncSetAttribute(consensus_fused_kernel<R, W>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  cudaError_t e = cudaFuncSetAttribute(consensus_fused_kernel<R, W, T>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        (int)smem);
   if (e != cudaSuccess) return e;
-  e = cudaFuncSetAttribute(consensus_fused_kernel<R, W>, cudaFuncAttributePreferredSharedMemoryCarveout,
+  e = cudaFuncSetAttribute(consensus_fused_kernel<R, W, T>, cudaFuncAttributePreferredSharedMemoryCarveout,
                            cudaSharedmemCarveoutMaxShared);
   if (e != cudaSuccess) return e;
   const int64_t tiles = (d + W - 1) / W;
-  consensus_fused_kernel<R, W><<<(unsigned)tiles, kFusedThreads, smem, stream>>>(mxi, myi, mxo, myo, args);
+  consensus_fused_kernel<R, W, T><<<(unsigned)tiles, T, smem, stream>>>(mxi, myi, mxo, myo, args);
   return cudaGetLastError();
 }
 
@@ -338,18 +338,17 @@ static ceca_status_t consensus_fused(const float *X, const float *Y, float *Xo, 
   cudaError_t e;
   if (tile_cols == kWideTileCols) {
     const int rows_per_thread = (n + 63) / 64;  // 64 row groups; n <= 256 -> at most 4
-    if (rows_per_thread <= 1)      e = launch_fused<1, kWideTileCols>(mxi, myi, mxo, myo, args, d, stream);
-    else if (rows_per_thread <= 2) e = launch_fused<2, kWideTileCols>(mxi, myi, mxo, myo, args, d, stream);
-    else if (rows_per_thread <= 3) e = launch_fused<3, kWideTileCols>(mxi, myi, mxo, myo, args, d, stream);
-    else                           e = launch_fused<4, kWideTileCols>(mxi, myi, mxo, myo, args, d, stream);
+    if (rows_per_thread <= 1)      e = launch_fused<1, kWideTileCols, kFusedThreads>(mxi, myi, mxo, myo, args, d, stream);
+    else if (rows_per_thread <= 2) e = launch_fused<2, kWideTileCols, kFusedThreads>(mxi, myi, mxo, myo, args, d, stream);
+    else if (rows_per_thread <= 3) e = launch_fused<3, kWideTileCols, kFusedThreads>(mxi, myi, mxo, myo, args, d, stream);
+    else                           e = launch_fused<4, kWideTileCols, kFusedThreads>(mxi, myi, mxo, myo, args, d, stream);
   } else {
-    const int rows_per_thread = (n + 255) / 256;  // 256 row groups; n <= 2048 -> at most 8
-    if (rows_per_thread <= 2)      e = launch_fused<2, kNarrowTileCols>(mxi, myi, mxo, myo, args, d, stream);
-    else if (rows_per_thread <= 3) e = launch_fused<3, kNarrowTileCols>(mxi, myi, mxo, myo, args, d, stream);
-    else if (rows_per_thread <= 4) e = launch_fused<4, kNarrowTileCols>(mxi, myi, mxo, myo, args, d, stream);
-    else if (rows_per_thread <= 5) e = launch_fused<5, kNarrowTileCols>(mxi, myi, mxo, myo, args, d, stream);
-    else if (rows_per_thread <= 6) e = launch_fused<6, kNarrowTileCols>(mxi, myi, mxo, myo, args, d, stream);
-    else                           e = launch_fused<8, kNarrowTileCols>(mxi, myi, mxo, myo, args, d, stream);
+    constexpr int kNarrowThreads = 512;  // one row group per thread: more warps per SM for the exchange loop
+    const int rows_per_thread = (n + kNarrowThreads - 1) / kNarrowThreads;  // n <= 2048 -> at most 4
+    if (rows_per_thread <= 1)      e = launch_fused<1, kNarrowTileCols, kNarrowThreads>(mxi, myi, mxo, myo, args, d, stream);
+    else if (rows_per_thread <= 2) e = launch_fused<2, kNarrowTileCols, kNarrowThreads>(mxi, myi, mxo, myo, args, d, stream);
+    else if (rows_per_thread <= 3) e = launch_fused<3, kNarrowTileCols, kNarrowThreads>(mxi, myi, mxo, myo, args, d, stream);
+    else                           e = launch_fused<4, kNarrowTileCols, kNarrowThreads>(mxi, myi, mxo, myo, args, d, stream);
   }
   return e == cudaSuccess ? CECA_OK : CECA_ERR_CUDA;
 }
