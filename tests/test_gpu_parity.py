@@ -323,6 +323,47 @@ def test_fused_consensus_padded_rows():
         assert ceca.ceca_read_status(ws) == 0
 
 
+def test_step_and_consensus_on_random_shapes():
+    """Seeded random draw of agent counts, widths, paddings, base offsets, iteration counters and call
+    forms (in / out of place, with / without gradient, fused / per round)."""
+    rng = np.random.default_rng(2024)
+    for case in range(80):
+        n = int(rng.choice([rng.integers(1, 9), rng.integers(9, 130), rng.integers(130, 700)]))
+        d = int(rng.choice([rng.integers(1, 9), rng.integers(9, 300), rng.integers(300, 3000)]))
+        ld = d + int(rng.choice([0, 0, 1, 3, 4, 28]))
+        offset = int(rng.choice([0, 0, 4, 1]))
+        variant = ceca.CECA_2P if (n % 2 and n > 1) else int(rng.choice([ceca.CECA_1P, ceca.CECA_2P]))
+        k = int(rng.integers(0, 2**50))
+        gamma = float(rng.choice([0.0, 0.05, 1.0]))
+        with_g = bool(rng.integers(0, 2))
+        x, y, g = synth.step_inputs(n, d, seed=case, x_std=1.0, g_std=1.0, same_xy=False)
+        (X, _), (Y, _) = _put(x.to(DEV), ld, offset), _put(y.to(DEV), ld, offset)
+        G = _put(g.to(DEV), ld, offset)[0] if with_g else None
+        want_x, want_y = oracle.step(_np(x), _np(y), _np(g) if with_g else None, np.float32(gamma), variant, k)
+        tol = STEP_TOL * _scale(gamma, (x, 1), (y, 1), (g if with_g else None, gamma))
+        if rng.integers(0, 2):
+            ceca.ceca_gossip_sgd_step(X, Y, G, gamma, variant, k)
+            Xo, Yo = X, Y
+        else:
+            (Xo, _), (Yo, _) = _padded(n, d, ld, offset), _padded(n, d, ld, offset)
+            ceca.ceca_gossip_sgd_step(X, Y, G, gamma, variant, k, X_out=Xo, Y_out=Yo)
+        assert np.abs(_np(Xo) - want_x).max() <= tol, (case, n, d, ld, offset, variant, k)
+        assert np.abs(_np(Yo) - want_y).max() <= tol, (case, n, d, ld, offset, variant, k)
+        # consensus from the same data: a few rounds from a random start, fused where the layout allows
+        rounds = int(rng.integers(1, 14))
+        k0 = int(rng.integers(0, 40))
+        ld4 = (d + 3) // 4 * 4 + 4 * int(rng.integers(0, 3))
+        (Xc, _), (Yc, _) = _put(x.to(DEV), ld4, 0), _put(y.to(DEV), ld4, 0)
+        fused = int(n <= 2048 and rng.integers(0, 2))
+        ws = _fused_ws()
+        ceca.ceca_consensus_rounds(Xc, Yc, variant, k0, rounds, fused, workspace=ws)
+        assert ceca.ceca_read_status(ws) == 0
+        want_x, want_y = oracle.consensus(_np(x), _np(y), variant, k0, rounds)
+        tol = STEP_TOL * rounds * _scale(0, (x, 1), (y, 1))
+        assert np.abs(_np(Xc) - want_x).max() <= tol, (case, n, d, ld4, variant, k0, rounds, fused)
+        assert np.abs(_np(Yc) - want_y).max() <= tol, (case, n, d, ld4, variant, k0, rounds, fused)
+
+
 # --------------------------------------------------------------------------------------------
 # logistic gradient
 # --------------------------------------------------------------------------------------------
