@@ -110,7 +110,8 @@ ceca_status_t ceca_gossip_sgd_step(const float *X, const float *Y, const float *
  *              TMA (cp.async.bulk.tensor), every round runs on chip, and the tile is written
  *              back once.  Needs n <= 2048 (32-column tiles up to n = 256, 8-column tiles above),
  *              X / X_out (and Y / Y_out when used) 16-byte aligned
- *              with ld*4 a multiple of 16 (else CECA_ERR_ALIGNMENT), ld < 2^32, rounds <= 64,
+ *              with ld*4 a multiple of 16 (else CECA_ERR_ALIGNMENT), ld < 2^32 (more than 64 rounds
+ *              run as several launches and then need Y_out),
  *              and a workspace of ceca_workspace_bytes(CECA_WS_CONSENSUS_FUSED, ...) bytes
  *              whose first int32 is a status word: it is left unchanged when the launch
  *              completes normally and set non-zero if a bounded on-chip wait for a TMA

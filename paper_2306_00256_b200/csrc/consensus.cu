@@ -382,9 +382,20 @@ extern "C" ceca_status_t ceca_consensus_rounds(const float *X, const float *Y, f
     return e == cudaSuccess ? CECA_OK : CECA_ERR_CUDA;
   }
 
-  if (fused)
-    return consensus_fused(X, Y, X_out, Y_out, n, d, ld, variant, k0, rounds, workspace, workspace_bytes,
-                           stream);
+  if (fused) {
+    // the kernel takes at most kMaxFusedRounds rounds per launch: longer runs go in chunks, the
+    // first from the inputs to the outputs, the others in place on the outputs
+    if (rounds > kMaxFusedRounds && !Y_out) return CECA_ERR_UNSUPPORTED;  // Y has to live somewhere in between
+    const float *x_in = X, *y_in = Y;
+    for (int32_t done = 0; done < rounds; done += kMaxFusedRounds) {
+      const int32_t chunk = rounds - done < kMaxFusedRounds ? rounds - done : kMaxFusedRounds;
+      st = consensus_fused(x_in, y_in, X_out, Y_out, n, d, ld, variant, k0 + done, chunk, workspace,
+                           workspace_bytes, stream);
+      if (st != CECA_OK) return st;
+      x_in = X_out; y_in = Y_out;
+    }
+    return CECA_OK;
+  }
 
   if (!Y && first.reads_y) return CECA_ERR_INVALID_ARG;
   float *y_work = Y_out;

@@ -309,6 +309,23 @@ def test_consensus_optional_y(fused):
     assert torch.equal(oc, one)
 
 
+def test_fused_consensus_many_rounds():
+    """More rounds than one launch takes: chunks of 64, continuing in place."""
+    n, d, rounds, k0 = 12, 200, 150, 5
+    x = synth.consensus_inputs(n, d, seed=3)
+    y = synth.consensus_inputs(n, d, seed=4, offset_rows=False)
+    for variant in (ceca.CECA_2P, ceca.CECA_1P):
+        Xo, Yo = torch.empty(n, d, device=DEV), torch.empty(n, d, device=DEV)
+        ws = _fused_ws()
+        ceca.ceca_consensus_rounds(x.to(DEV), y.to(DEV), variant, k0, rounds, 1, X_out=Xo, Y_out=Yo, workspace=ws)
+        assert ceca.ceca_read_status(ws) == 0
+        want_x, want_y = oracle.consensus(_np(x), _np(y), variant, k0, rounds)
+        tol = STEP_TOL * rounds * _scale(0, (x, 1), (y, 1))
+        assert np.abs(_np(Xo) - want_x).max() <= tol and np.abs(_np(Yo) - want_y).max() <= tol
+        with pytest.raises(ceca.CecaError):   # nowhere to keep Y between the launches
+            ceca.ceca_consensus_rounds(x.to(DEV), y.to(DEV), variant, k0, rounds, 1, X_out=Xo, workspace=ws, want_y=False)
+
+
 def test_fused_consensus_padded_rows():
     n, d, ld = 100, 1000, 1024
     x = synth.consensus_inputs(n, d, seed=9)
