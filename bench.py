@@ -161,6 +161,16 @@ def oracle_step_throughput(n, variant, gamma, cols, steps, threads=None):
     return n * cols * steps / dt, dt / steps, threads
 
 
+def cpu_model():
+    try:
+        for line in open("/proc/cpuinfo"):
+            if line.startswith("model name"):
+                return line.split(":", 1)[1].strip()
+    except OSError:
+        pass
+    return "unknown"
+
+
 def run_reference(args, wl, rank, world):
     """--impl reference: the fp64 oracle, as it stands, on the host cores, on a column slice."""
     if rank != 0:
@@ -177,7 +187,8 @@ def run_reference(args, wl, rank, world):
             "vs_baseline": None, "dtype": "f64", "data": "synthetic",
             "config": {"workload": args.workload, "n_agents": wl["n"], "d": wl["d"], "variant": "2P" if wl["variant"] == 2 else "1P",
                        "sample_columns": cols},
-            "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample,
+                             "host_cores": os.cpu_count(), "cpu_model": cpu_model()},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
     print(json.dumps(line))
 
@@ -533,8 +544,10 @@ def main():
     if rank == 0 and world == 1 and wl["kind"] == "step" and not args.no_cpu_baseline:
         cols = min(wl["d"], 262_144)
         v, sec, threads = oracle_step_throughput(wl["n"], wl["variant"], wl["gamma"], cols, 3 * extra["tau"])
+        v1, _, _ = oracle_step_throughput(wl["n"], wl["variant"], wl["gamma"], cols // 4, extra["tau"], threads=1)
         cpu = {"value": v, "unit": UNIT, "cores": threads, "kind": "oracle",
-               "sample": "%d-column slice (all %d rows), %d steps = 3 cycles of the CECA sequence, fp64" % (cols, wl["n"], 3 * extra["tau"])}
+               "sample": "%d-column slice (all %d rows), %d steps = 3 cycles of the CECA sequence, fp64" % (cols, wl["n"], 3 * extra["tau"]),
+               "single_thread_value": v1, "host_cores": os.cpu_count(), "cpu_model": cpu_model()}
 
     if rank == 0:
         config = {"workload": args.workload, "n_agents": wl["n"], "d": wl["d"], "variant": "2P" if wl["variant"] == 2 else "1P"}
