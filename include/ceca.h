@@ -91,6 +91,10 @@ ceca_status_t ceca_schedule(int32_t n, ceca_variant_t variant, int64_t k, ceca_r
  * x, and X never depends on Y (CECA-2P is then the one-peer exponential graph).  Passing Y == NULL
  * and Y_out == NULL runs just the x update: 12 bytes per agent-parameter instead of 20.  For any
  * other n this combination is CECA_ERR_INVALID_ARG.
+ * Dead-y form: in the last round of a cycle (r = tau-1) the new y is never used, because round 0 has
+ * b = 0 and builds its message from x (Algorithm 1 with n_0 = 0).  Passing Y_out == NULL there (with Y
+ * given) skips that write: 16 bytes per agent-parameter; the caller's Y buffer keeps its old contents
+ * until round 0 overwrites it.  Y_out == NULL with Y given in any other round is CECA_ERR_INVALID_ARG.
  * fp32 arithmetic; a, b and 1-a, 1-b are formed in fp64 on the host and rounded once.
  */
 ceca_status_t ceca_gossip_sgd_step(const float *X, const float *Y, const float *G, float *X_out,

@@ -119,12 +119,13 @@ def ceca_schedule(n, variant, k, peers=True):
     return rd, recv, send
 
 
-def ceca_gossip_sgd_step(X, Y, G, gamma, variant, k, X_out=None, Y_out=None, stream=None):
+def ceca_gossip_sgd_step(X, Y, G, gamma, variant, k, X_out=None, Y_out=None, stream=None, drop_y=False):
     """One DSGD-CECA iteration on device tensors.  Outputs default to in place.  Returns (X_out, Y_out).
-    Y = Y_out = None asks for the X-only update (n a power of two)."""
+    Y = Y_out = None asks for the X-only update (n a power of two); drop_y=True passes Y_out = NULL
+    with Y given (legal in the last round of a cycle, where the new y is never used)."""
     n, d, ld = _matrix(X, "X")
     X_out = X if X_out is None else X_out
-    if Y_out is None and Y is not None:
+    if Y_out is None and Y is not None and not drop_y:
         Y_out = Y   # (Y and Y_out both None: the X-only update, legal for n a power of two)
     for t, name in ((Y, "Y"), (G, "G"), (X_out, "X_out"), (Y_out, "Y_out")):
         if t is not None and _matrix(t, name, n) != (n, d, ld):

@@ -69,10 +69,12 @@ struct RowRegs {
 // thread); MINB = CTAs per SM the register allocation must allow (parallelism across threads).
 // Long cycles want a deep RIF, cycles of two rows have only two rows to load and want occupancy.
 // YMODE: 1 = Y is read and written; 0 = Y has zero weight this round, it is only written;
-//        2 = X only (n a power of two: every round builds its message from x, so X never depends on Y).
+//        2 = X only (n a power of two: every round builds its message from x, so X never depends on Y);
+//        3 = Y is read but y+ is not stored (last round of a cycle: the next round ignores y).
 template <typename V, bool HAS_G, int YMODE, int RIF, int MINB>
 __global__ void __launch_bounds__(kThreads, MINB) step_walk_kernel(const StepArgs p) {
-  constexpr bool USE_Y = (YMODE == 1);
+  constexpr bool USE_Y = (YMODE == 1 || YMODE == 3);
+  constexpr bool WRITE_Y = (YMODE == 0 || YMODE == 1);
   constexpr int VW = sizeof(V) / sizeof(float);
   const int64_t colv = (int64_t)blockIdx.x * kThreads + threadIdx.x;
   if (colv >= p.ncolv) return;
@@ -110,7 +112,7 @@ __global__ void __launch_bounds__(kThreads, MINB) step_walk_kernel(const StepArg
           V own_x, own_y, u;
           batch[j].own_terms(p, own_x, own_y, u);
           vstore<V>(p.Xo + offs[j], vfma(p.a, own_x, vmul(p.one_minus_a, u_prev)));
-          if (YMODE != 2) vstore<V>(p.Yo + offs[j], vfma(p.b, own_y, vmul(p.one_minus_b, u_prev)));
+          if (WRITE_Y) vstore<V>(p.Yo + offs[j], vfma(p.b, own_y, vmul(p.one_minus_b, u_prev)));
           u_prev = u;
         }
       }
@@ -118,7 +120,7 @@ __global__ void __launch_bounds__(kThreads, MINB) step_walk_kernel(const StepArg
     if (!first_done) first.own_terms(p, first_own_x, first_own_y, u_prev);  // cycle of one row
     // close the cycle: the first row receives the message of the last one
     vstore<V>(p.Xo + first_off, vfma(p.a, first_own_x, vmul(p.one_minus_a, u_prev)));
-    if (YMODE != 2) vstore<V>(p.Yo + first_off, vfma(p.b, first_own_y, vmul(p.one_minus_b, u_prev)));
+    if (WRITE_Y) vstore<V>(p.Yo + first_off, vfma(p.b, first_own_y, vmul(p.one_minus_b, u_prev)));
   }
 }
 
@@ -130,11 +132,13 @@ static cudaError_t launch_walk_shape(const StepArgs &args, bool has_g, int ymode
   if (has_g) {
     if (ymode == 1)      step_walk_kernel<V, true, 1, RIF, MINB><<<grid, kThreads, 0, stream>>>(args);
     else if (ymode == 0) step_walk_kernel<V, true, 0, RIF, MINB><<<grid, kThreads, 0, stream>>>(args);
-    else                 step_walk_kernel<V, true, 2, RIF, MINB><<<grid, kThreads, 0, stream>>>(args);
+    else if (ymode == 2) step_walk_kernel<V, true, 2, RIF, MINB><<<grid, kThreads, 0, stream>>>(args);
+    else                 step_walk_kernel<V, true, 3, RIF, MINB><<<grid, kThreads, 0, stream>>>(args);
   } else {
     if (ymode == 1)      step_walk_kernel<V, false, 1, RIF, MINB><<<grid, kThreads, 0, stream>>>(args);
     else if (ymode == 0) step_walk_kernel<V, false, 0, RIF, MINB><<<grid, kThreads, 0, stream>>>(args);
-    else                 step_walk_kernel<V, false, 2, RIF, MINB><<<grid, kThreads, 0, stream>>>(args);
+    else if (ymode == 2) step_walk_kernel<V, false, 2, RIF, MINB><<<grid, kThreads, 0, stream>>>(args);
+    else                 step_walk_kernel<V, false, 3, RIF, MINB><<<grid, kThreads, 0, stream>>>(args);
   }
   return cudaGetLastError();
 }
@@ -146,7 +150,7 @@ template <typename V>
 static cudaError_t launch_walk(const StepArgs &args, bool has_g, int ymode, cudaStream_t stream) {
   if (args.ncolv <= 0) return cudaSuccess;
   if (args.cycle_len <= 2)
-    return ymode == 1 ? launch_walk_shape<V, 1, 4>(args, has_g, ymode, stream)
+    return (ymode == 1 || ymode == 3) ? launch_walk_shape<V, 1, 4>(args, has_g, ymode, stream)
                       : launch_walk_shape<V, 1, 6>(args, has_g, ymode, stream);
   if (args.cycle_len <= 4) return launch_walk_shape<V, 2, 4>(args, has_g, ymode, stream);
   return launch_walk_shape<V, 4, 2>(args, has_g, ymode, stream);
@@ -154,8 +158,8 @@ static cudaError_t launch_walk(const StepArgs &args, bool has_g, int ymode, cuda
 
 static inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
-// Enqueues one iteration.  Arguments are assumed validated.  Yo == nullptr selects the X-only update
-// (the caller has checked that n is a power of two).
+// Enqueues one iteration.  Arguments are assumed validated.  Yo == nullptr: y+ is not stored (the
+// caller has checked that this is legal); Y is then still read if the round needs it.
 cudaError_t enqueue_step(const Plan &plan, const float *X, const float *Y, const float *G, float *Xo,
                          float *Yo, int32_t n, int64_t d, int64_t ld, float gamma,
                          cudaStream_t stream) {
@@ -168,8 +172,8 @@ cudaError_t enqueue_step(const Plan &plan, const float *X, const float *Y, const
   a.a = plan.a; a.b = plan.b; a.one_minus_a = plan.one_minus_a; a.one_minus_b = plan.one_minus_b;
   a.gamma = gamma;
   const bool has_g = (G != nullptr);
-  const int ymode = !Yo ? 2 : (plan.reads_y ? 1 : 0);
-  const bool use_y = (ymode == 1);
+  const int ymode = Yo ? (plan.reads_y ? 1 : 0) : ((Y && plan.reads_y) ? 3 : 2);
+  const bool use_y = (ymode == 1 || ymode == 3);
   const bool vec_ok = (ld % 4 == 0) && aligned16(X) && aligned16(Xo) && (!Yo || aligned16(Yo)) &&
                       (!use_y || aligned16(Y)) && (!has_g || aligned16(G));
   const int64_t d_vec = vec_ok ? (d / 4) * 4 : 0;  // columns covered by 128-bit accesses
@@ -208,8 +212,12 @@ extern "C" ceca_status_t ceca_gossip_sgd_step(const float *X, const float *Y, co
   st = ceca::make_plan(n, variant, k, &plan);
   if (st != CECA_OK) return st;
   if (!Y_out) {
-    // X-only update: legal exactly when no round ever builds its message from y, i.e. n-1 is all ones
-    if (Y || (n & (n - 1)) != 0) return CECA_ERR_INVALID_ARG;
+    // y+ may be dropped in two situations: n-1 is all ones (no round ever builds its message from y,
+    // so Y is not needed at all), or this is the last round of a cycle (round 0 ignores y and
+    // overwrites it)
+    const bool power_of_two = (n & (n - 1)) == 0;
+    const bool last_round = plan.rd.tau > 0 && plan.rd.r == plan.rd.tau - 1;
+    if (!(Y ? last_round : power_of_two)) return CECA_ERR_INVALID_ARG;
   } else if (!Y && plan.reads_y) {
     return CECA_ERR_INVALID_ARG;
   }

@@ -187,6 +187,31 @@ def test_x_only_step_for_power_of_two_agents(n, d):
             ceca.ceca_gossip_sgd_step(bad, None, None, gamma, ceca.CECA_2P, 0, X_out=torch.empty_like(bad))
 
 
+@pytest.mark.parametrize("n,variant", [(2, ceca.CECA_2P), (5, ceca.CECA_2P), (6, ceca.CECA_1P), (24, ceca.CECA_1P),
+                                       (97, ceca.CECA_2P), (100, ceca.CECA_2P)])
+def test_dead_y_may_be_dropped_in_the_last_round_of_a_cycle(n, variant):
+    """Round tau-1 without storing y+, then round 0: the same X and Y bits as the full updates, because
+    round 0 has b = 0 and builds its message from x."""
+    d, gamma = 1029, 0.1
+    tau = _tau(n)
+    x, y, g = synth.step_inputs(n, d, seed=n, x_std=1.0, g_std=1.0, same_xy=False)
+    g2 = synth.gradient_inputs(n, d, 1, g_std=1.0)
+    k = 3 * tau + tau - 1
+    Xf, Yf = x.to(DEV), y.to(DEV)                        # full path
+    ceca.ceca_gossip_sgd_step(Xf, Yf, g.to(DEV), gamma, variant, k)
+    Xl, Yl = x.to(DEV), y.to(DEV)                        # y+ dropped
+    ceca.ceca_gossip_sgd_step(Xl, Yl, g.to(DEV), gamma, variant, k, drop_y=True)
+    assert torch.equal(Xl, Xf) and torch.equal(Yl.cpu(), y)   # X as in the full update, Y untouched
+    want_x, _ = oracle.step(_np(x), _np(y), _np(g), np.float32(gamma), variant, k)
+    assert np.abs(_np(Xl) - want_x).max() <= STEP_TOL * _scale(gamma, (x, 1), (y, 1), (g, gamma))
+    ceca.ceca_gossip_sgd_step(Xf, Yf, g2.to(DEV), gamma, variant, k + 1)
+    ceca.ceca_gossip_sgd_step(Xl, Yl, g2.to(DEV), gamma, variant, k + 1)
+    assert torch.equal(Xl, Xf) and torch.equal(Yl, Yf)
+    if tau > 1:
+        with pytest.raises(ceca.CecaError):
+            ceca.ceca_gossip_sgd_step(Xl, Yl, g.to(DEV), gamma, variant, k + 1, drop_y=True)
+
+
 @pytest.mark.parametrize("n,variant", [(5, ceca.CECA_2P), (6, ceca.CECA_1P), (63, ceca.CECA_2P), (64, ceca.CECA_1P)])
 def test_mean_lemma_and_resume_on_gpu(n, variant):
     """Lemma "relation between averaged variables": with x0 = y0 the mean takes a plain SGD step.

@@ -87,7 +87,7 @@ def test_device_entry_points_reject_bad_arguments_before_touching_the_gpu():
     assert step(fake, None, fake, fake, ctypes.c_void_p(512), 4, 8, 8, 0.1, 2, 1, None) == 1  # round 1 needs Y
     assert step(fake, fake, None, fake, fake, 4, 8, 8, 0.1, 2, 1, None) == 4      # X_out == Y_out
     assert step(fake, None, fake, ctypes.c_void_p(512), None, 6, 8, 8, 0.1, 2, 0, None) == 1   # X-only needs n = 2^tau
-    assert step(fake, fake, fake, ctypes.c_void_p(512), None, 8, 8, 8, 0.1, 2, 0, None) == 1   # ... and no Y at all
+    assert step(fake, fake, fake, ctypes.c_void_p(512), None, 8, 8, 8, 0.1, 2, 0, None) == 1   # y+ may only be dropped at r = tau-1
     cons = lib.ceca_consensus_rounds
     assert cons(fake, fake, fake, fake, 4, 8, 8, 2, 0, -1, 0, None, 0, None) == 1
     assert cons(fake, None, ctypes.c_void_p(512), None, 4, 8, 8, 2, 0, 2, 0, None, 0, None) == 5  # no Y_out, no workspace
