@@ -163,6 +163,16 @@ def oracle_step_throughput(n, variant, gamma, cols, steps, threads=None):
     return n * cols * steps / dt, dt / steps, threads
 
 
+def host_memory_available():
+    try:
+        for line in open("/proc/meminfo"):
+            if line.startswith("MemAvailable"):
+                return int(line.split()[1]) * 1024
+    except OSError:
+        pass
+    return None
+
+
 def cpu_model():
     try:
         for line in open("/proc/cpuinfo"):
@@ -538,8 +548,15 @@ def main():
 
     e2e = None
     if wl["kind"] == "step" and not args.no_e2e and not wl.get("x_only") and not wl.get("drop_dead_y"):
-        e2e = bench_step_e2e(args, wl, device)
-        if dist is not None:
+        need = world * 3 * units_per_step * 4          # every rank keeps X, Y, G of its block in host memory
+        avail = host_memory_available()
+        if avail is not None and need > 0.7 * avail:
+            e2e = {"value": None, "unit": UNIT, "h2d_bytes_per_step": None, "d2h_bytes_per_step": None,
+                   "unavailable": "host buffers for %d ranks need %.0f GB, the host has %.0f GB available" % (
+                       world, need / 1e9, avail / 1e9)}
+        else:
+            e2e = bench_step_e2e(args, wl, device)
+        if dist is not None and e2e.get("value") is not None:
             ms = max_over_ranks(e2e["ms_per_step"], dist, device)
             e2e["ms_per_step"] = ms
             e2e["value"] = world * units_per_step / (ms * 1e-3)
