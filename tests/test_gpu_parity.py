@@ -121,6 +121,20 @@ def test_consensus_at_the_papers_network_sizes(n, variant):
     assert np.abs(_np(X) - want_x).max() <= tol and np.abs(_np(Y) - want_y).max() <= tol
 
 
+def test_step_with_more_cycles_than_one_grid_dimension_holds():
+    """140,000 agents: the 1-port matching has 70,000 cycles (more than 65,535 grid rows), and the
+    2-port shift n/2 as well."""
+    n, d, gamma = 140_000, 5, 0.1
+    x, y, g = synth.step_inputs(n, d, seed=1, x_std=1.0, g_std=1.0, same_xy=False)
+    tau = _tau(n)
+    tol = STEP_TOL * _scale(gamma, (x, 1), (y, 1), (g, gamma))
+    for variant, k in [(ceca.CECA_1P, 0), (ceca.CECA_1P, tau - 1), (ceca.CECA_2P, 1), (ceca.CECA_2P, tau - 1)]:
+        X, Y, G = x.to(DEV), y.to(DEV), g.to(DEV)
+        ceca.ceca_gossip_sgd_step(X, Y, G, gamma, variant, k)
+        want_x, want_y = oracle.step(_np(x), _np(y), _np(g), np.float32(gamma), variant, k)
+        assert np.abs(_np(X) - want_x).max() <= tol and np.abs(_np(Y) - want_y).max() <= tol, (variant, k)
+
+
 @pytest.mark.parametrize("n,d,ld,offset", [(6, 37, 40, 0), (6, 37, 41, 0), (24, 1000, 1024, 4), (24, 1000, 1024, 1),
                                            (97, 513, 517, 3), (100, 4096, 4100, 0)])
 def test_step_padded_rows_and_unaligned_bases(n, d, ld, offset):
