@@ -623,26 +623,28 @@ def test_full_size_consensus_on_column_windows(fused):
         assert np.abs(_np(Yo[:, lo:hi]) - want_y).max() <= tol
 
 
-def test_heterogeneous_logreg_full_size_first_iterations():
-    """n = 63, 2000 samples, d = 4096, per-agent feature shifts: gradient + fused step, 2-port, checked
-    against the oracle for the first iterations."""
-    n, m, d, gamma = 63, 2000, 4096, 0.01
+@pytest.mark.parametrize("n,variant", [(63, ceca.CECA_2P), (62, ceca.CECA_1P), (64, ceca.CECA_1P)])
+def test_heterogeneous_logreg_full_size_first_iterations(n, variant):
+    """2000 samples per agent, d = 4096, per-agent feature shifts: gradient + fused step, checked against
+    the oracle for the first iterations (a full CECA cycle and one more, so that rounds that evaluate the
+    gradient at y are included).  The 1-port variant needs an even n: 62 and 64 stand beside n = 63."""
+    m, d, gamma = 2000, 4096, 0.01
     _need_free(int(1.3 * n * m * d * 4))
     A, L, _ = synth.logreg_problem(n, m, d, seed=3, flip=0.05, hetero_std=0.5, device=DEV)
     X = torch.zeros(n, d, device=DEV); Y = torch.zeros(n, d, device=DEV); G = torch.empty(n, d, device=DEV)
     ws = torch.empty(ceca.ceca_workspace_bytes(ceca.WS_LOGREG_GRAD, n, m, d) // 4, dtype=torch.float32, device=DEV)
-    agents = [0, 31, 62]
+    agents = [0, n // 2, n - 1]
     an = {i: _np(A[i:i + 1]) for i in agents}
     ln = {i: _np(L[i:i + 1]) for i in agents}
-    for k in range(4):
-        ceca.dsgd_logreg_grad(A, L, X, Y, k, ceca.CECA_2P, G, ws)
+    for k in range(_tau(n) + 1):
+        ceca.dsgd_logreg_grad(A, L, X, Y, k, variant, G, ws)
         z = Y if oracle.round_info(n, k).payload else X
         for i in agents:   # the gradient of agent i depends on its own data and model only
             zi = _np(z[i:i + 1])
             want = oracle.logreg_grad(an[i], ln[i], zi, zi, 0)
             assert np.abs(_np(G[i:i + 1]) - want).max() <= _grad_tol(d, want), (k, i)
         bx, by, bg = _np(X), _np(Y), _np(G)
-        ceca.ceca_gossip_sgd_step(X, Y, G, gamma, ceca.CECA_2P, k)
-        want_x, want_y = oracle.step(bx, by, bg, np.float32(gamma), ceca.CECA_2P, k)
+        ceca.ceca_gossip_sgd_step(X, Y, G, gamma, variant, k)
+        want_x, want_y = oracle.step(bx, by, bg, np.float32(gamma), variant, k)
         tol = STEP_TOL * max(np.abs(bx).max(), np.abs(by).max(), gamma * np.abs(bg).max())
         assert np.abs(_np(X) - want_x).max() <= tol and np.abs(_np(Y) - want_y).max() <= tol
