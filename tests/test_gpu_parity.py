@@ -448,6 +448,36 @@ def test_logreg_grad_matches_oracle(n, m, d):
             assert torch.equal(G, G2)  # run-to-run identical
 
 
+@pytest.mark.parametrize("n,m,d,ld", [(6, 40, 512, 516), (6, 40, 512, 513), (3, 33, 2052, 2080), (5, 50, 10, 12)])
+def test_gradients_with_padded_rows_leave_padding_and_workspace_guard_alone(n, m, d, ld):
+    """X, Y, G (and the least-squares noise) with ld > d; the columns between d and ld of G, and a guard
+    area behind the stated workspace size, must keep their canary values."""
+    a, lab, _ = synth.logreg_problem(n, m, d, seed=n + d, flip=0.1, hetero_std=0.3)
+    a2, b2, _ = synth.lsq_problem(n, m, d, seed=n + d + 1)
+    gen = torch.Generator().manual_seed(7)
+    x = 0.1 * torch.randn(n, d, generator=gen); y = 0.1 * torch.randn(n, d, generator=gen)
+    eps = synth.gradient_noise(n, d, 0, sigma_n=1.0)
+    (X, _), (Y, _), (E, _) = _put(x.to(DEV), ld), _put(y.to(DEV), ld), _put(eps.to(DEV), ld)
+    need = ceca.ceca_workspace_bytes(ceca.WS_LOGREG_GRAD, n, m, d)
+    assert need % 4 == 0
+    guard = 1024
+    ws_all = torch.full((need // 4 + guard,), float("nan"), dtype=torch.float32, device=DEV)
+    ws = ws_all[:need // 4]
+    for k in range(_tau(n)):
+        G, gbuf = _padded(n, d, ld)
+        ceca.dsgd_logreg_grad(a.to(DEV), lab.to(DEV), X, Y, k, ceca.CECA_2P, G, ws)
+        want = oracle.logreg_grad(_np(a), _np(lab), _np(x), _np(y), k)
+        assert np.abs(_np(G) - want).max() <= _grad_tol(d, want)
+        assert torch.isnan(gbuf[:n * ld].view(n, ld)[:, d:]).all() and torch.isnan(gbuf[n * ld:]).all()
+        G2, gbuf2 = _padded(n, d, ld)
+        ceca.dsgd_lsq_grad(a2.to(DEV), b2.to(DEV), X, Y, k, ceca.CECA_2P, G2, ws, noise=E)
+        want = oracle.lsq_grad(_np(a2), _np(b2), _np(x), _np(y), k, noise=_np(eps))
+        z = y if oracle.round_info(n, k).payload else x
+        assert np.abs(_np(G2) - want).max() <= _lsq_tol(_np(a2), _np(b2), _np(z)) + 5e-6
+        assert torch.isnan(gbuf2[:n * ld].view(n, ld)[:, d:]).all()
+        assert torch.isnan(ws_all[need // 4:]).all()
+
+
 @pytest.mark.parametrize("n,variant", [(5, ceca.CECA_2P), (6, ceca.CECA_1P)])
 def test_small_logistic_regression_run(n, variant):
     """n agents, d = 32, 100 samples each, X0 = Y0 = 0, gamma = 0.05, 60 iterations: gradient kernel
