@@ -264,7 +264,8 @@ def bench_step(args, wl, device, dist):
         roof = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                 "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH.get(args.workload),
                 "kernel": "step_walk_kernel<float4, gradient, %s>" % ("X only" if x_only else "reads Y"), "peak_source": "of " + which,
-                "avg_launch_ms": avg_ms, "launches_timed": len(dominant),
+                "avg_launch_ms": avg_ms, "median_launch_ms": statistics.median(dominant), "best_launch_ms": min(dominant),
+                "launches_timed": len(dominant),
                 "frac_of_nominal_8TBs": achieved / 8000.0,
                 "ms_by_round": [round(statistics.mean(per_launch[s] for s in range(args.steps) if (k_first + s) % tau == r), 4)
                                 if any((k_first + s) % tau == r for s in range(args.steps)) else None for r in range(tau)]}
