@@ -317,6 +317,28 @@ def test_fused_consensus_above_256_agents(n, d):
             assert torch.equal(X, Xo) and torch.equal(Y, Yo)
 
 
+def test_finite_time_consensus_for_every_network_size():
+    """Sec. 5 "Finite-time exact consensus": for every n the residue sum_i ||x_i - mean|| is still large after
+    tau - 1 rounds and at rounding level after tau = ceil(log2 n) rounds (fused kernel, random x and y)."""
+    d = 96
+    for n in range(2, 141):
+        x = synth.consensus_inputs(n, d, seed=n, offset_rows=False)
+        y = synth.consensus_inputs(n, d, seed=n + 7, offset_rows=False)
+        mean = x.double().mean(0)
+        tau = _tau(n)
+        assert tau == int(np.ceil(np.log2(n)))
+        for variant in _variants(n):
+            ws = _fused_ws()
+            for rounds, reached in ((tau - 1, False), (tau, True)):
+                if rounds == 0:
+                    continue
+                Xo, Yo = torch.empty(n, d, device=DEV), torch.empty(n, d, device=DEV)
+                ceca.ceca_consensus_rounds(x.to(DEV), y.to(DEV), variant, 0, rounds, 1, X_out=Xo, Y_out=Yo, workspace=ws)
+                residue = float((Xo.double().cpu() - mean).norm(dim=1).sum()) / n
+                assert (residue < 1e-5) == reached, (n, variant, rounds, residue)
+            assert ceca.ceca_read_status(ws) == 0
+
+
 @pytest.mark.parametrize("fused", [0, 1])
 def test_consensus_optional_y(fused):
     n, d = 97, 1000
