@@ -109,7 +109,8 @@ ceca_status_t ceca_gossip_sgd_step(const float *X, const float *Y, const float *
  * consensus"); one more round makes Y_out the mean as well.
  *
  *   fused = 0: one kernel launch per round, each a full pass over HBM.  Works for every n, d,
- *              ld and alignment.  Y_out == NULL is allowed when workspace holds n*ld floats.
+ *              ld and alignment.  Y_out == NULL is allowed when workspace holds n*ld floats, and
+ *              without any workspace when n is a power of two (J then never feeds I).
  *   fused = 1: a single launch.  A column tile of all n rows is brought into shared memory by
  *              TMA (cp.async.bulk.tensor), every round runs on chip, and the tile is written
  *              back once.  Needs n <= 2048 (32-column tiles up to n = 256, 8-column tiles above),

@@ -397,6 +397,20 @@ extern "C" ceca_status_t ceca_consensus_rounds(const float *X, const float *Y, f
     return CECA_OK;
   }
 
+  if (!Y_out && (n & (n - 1)) == 0) {
+    // n a power of two and Y not wanted back: every round sends I, so J never matters; run the
+    // x-only form of the step kernel (8 bytes per element and round, no workspace)
+    const float *x_src = X;
+    for (int32_t t = 0; t < rounds; ++t) {
+      Plan plan;
+      st = make_plan(n, variant, k0 + t, &plan);
+      if (st != CECA_OK) return st;
+      if (enqueue_step(plan, x_src, nullptr, nullptr, X_out, nullptr, n, d, ld, 0.f, stream) != cudaSuccess)
+        return CECA_ERR_CUDA;
+      x_src = X_out;
+    }
+    return CECA_OK;
+  }
   if (!Y && first.reads_y) return CECA_ERR_INVALID_ARG;
   float *y_work = Y_out;
   if (!y_work) {  // the caller does not want Y back: keep it in the workspace

@@ -317,6 +317,21 @@ def test_fused_consensus_above_256_agents(n, d):
             assert torch.equal(X, Xo) and torch.equal(Y, Yo)
 
 
+@pytest.mark.parametrize("n", [2, 8, 64, 128])
+def test_per_round_consensus_without_y_for_power_of_two_agents(n):
+    """n = 2^tau and Y not wanted: no Y, no workspace, and the X of the full computation."""
+    d = 1003
+    x = synth.consensus_inputs(n, d, seed=n)
+    y = synth.consensus_inputs(n, d, seed=n + 1, offset_rows=False)
+    tau = _tau(n)
+    for variant in _variants(n):
+        for k0, rounds in [(0, tau), (2, tau + 3)]:
+            Xo = torch.full((n, d), float("nan"), device=DEV)
+            ceca.ceca_consensus_rounds(x.to(DEV), None, variant, k0, rounds, 0, X_out=Xo, want_y=False)
+            want_x, _ = oracle.consensus(_np(x), _np(y), variant, k0, rounds)
+            assert np.abs(_np(Xo) - want_x).max() <= STEP_TOL * rounds * float(x.abs().max()), (n, variant, k0)
+
+
 def test_finite_time_consensus_for_every_network_size():
     """Sec. 5 "Finite-time exact consensus": for every n the residue sum_i ||x_i - mean|| is still large after
     tau - 1 rounds and at rounding level after tau = ceil(log2 n) rounds (fused kernel, random x and y)."""

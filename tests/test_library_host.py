@@ -90,7 +90,7 @@ def test_device_entry_points_reject_bad_arguments_before_touching_the_gpu():
     assert step(fake, fake, fake, ctypes.c_void_p(512), None, 8, 8, 8, 0.1, 2, 0, None) == 1   # y+ may only be dropped at r = tau-1
     cons = lib.ceca_consensus_rounds
     assert cons(fake, fake, fake, fake, 4, 8, 8, 2, 0, -1, 0, None, 0, None) == 1
-    assert cons(fake, None, ctypes.c_void_p(512), None, 4, 8, 8, 2, 0, 2, 0, None, 0, None) == 5  # no Y_out, no workspace
+    assert cons(fake, None, ctypes.c_void_p(512), None, 6, 8, 8, 2, 0, 2, 0, None, 0, None) == 5  # no Y_out, no workspace (n not 2^tau)
     assert cons(fake, None, ctypes.c_void_p(512), None, 2050, 8, 8, 2, 0, 2, 1, fake, 256, None) == 4  # n > 2048 fused
     assert cons(fake, None, ctypes.c_void_p(516), None, 4, 8, 8, 2, 0, 2, 1, fake, 256, None) == 3  # misaligned
     assert cons(fake, None, ctypes.c_void_p(512), None, 4, 8, 6, 2, 0, 2, 1, fake, 256, None) == 1  # ld < d
