@@ -77,6 +77,11 @@ def test_schedule_errors():
 
 
 def test_device_entry_points_reject_bad_arguments_before_touching_the_gpu():
+    import torch
+    if torch.cuda.is_available():
+        # the stand-in pointers below must never reach a kernel; without a device a slip shows up as
+        # status 6 here, with a device it would be a fault, so this check only runs on CPU-only hosts
+        pytest.skip("argument-validation probe with stand-in pointers runs on CPU-only hosts")
     lib = ceca.library()
     fake = ctypes.c_void_p(256)  # never dereferenced: every call below fails validation first
     step = lib.ceca_gossip_sgd_step
