@@ -56,17 +56,17 @@ def test_static_scratch_gradient_matches_workspace_gradient_on_consecutive_calls
 
 @pytest.mark.gpu
 def test_static_scratch_rejects_problems_that_do_not_fit():
-    n, m, d = 64, 4000, 8192
+    n, m, d = 20, 1000, 8192     # needs ~41 MB of partial sums: more than the built-in 32 MiB
     cap = ceca.dsgd_logreg_grad_static_capacity()
     assert ceca.ceca_workspace_bytes(ceca.WS_LOGREG_GRAD, n, m, d) > cap
-    tiny = torch.zeros(16, device=DEV)
-    # the size check comes before anything touches the data, so small stand-in tensors are enough;
-    # the binding would object to their shapes, hence the raw call
-    lib = ceca.library()
-    st = lib.dsgd_logreg_grad_static(tiny.data_ptr(), tiny.data_ptr(), tiny.data_ptr(), tiny.data_ptr(), 0,
-                                     tiny.data_ptr(), n, m, d, d, ceca.CECA_2P, None)
-    assert st == 7 and "scratch" in ceca.ceca_status_string(st)
+    # real, full-size buffers: the call must return before touching them, but nothing is left to chance
+    A = torch.zeros(n, m, d, device=DEV); L = torch.ones(n, m, device=DEV)
+    X = torch.zeros(n, d, device=DEV); G = torch.full((n, d), 7.0, device=DEV)
+    with pytest.raises(ceca.CecaError) as err:
+        ceca.dsgd_logreg_grad_static(A, L, X, X, 0, ceca.CECA_2P, G)
+    assert err.value.status == 7 and "scratch" in str(err.value)
     torch.cuda.synchronize()
+    assert bool((G == 7.0).all())    # nothing was launched
 
 
 def test_static_scratch_capacity_is_stated():
