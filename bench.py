@@ -44,9 +44,13 @@ WORKLOADS = {
     "step_small": dict(kind="step", n=100, d=2_097_152, variant=2, gamma=0.1),
     # n a power of two: the X-only update (12 B per agent-parameter; CECA-2P = one-peer exponential graph)
     "pow2_xonly_step": dict(kind="step", n=128, d=8_388_608, variant=2, gamma=0.1, x_only=True),
+    # fused = 1 picks the kernel by n (tensor-memory exchange up to n = 128, shared-memory exchange above)
     "consensus_fused": dict(kind="consensus", n=97, d=1 << 20, variant=2, fused=1),
+    "consensus_fused_smem": dict(kind="consensus", n=97, d=1 << 20, variant=2, fused=2),
+    "consensus_fused_tmem": dict(kind="consensus", n=97, d=1 << 20, variant=2, fused=3),
     "consensus_rounds": dict(kind="consensus", n=97, d=1 << 20, variant=2, fused=0),
-    # the paper's larger network size (Sec. 5): 8-column tiles, eleven rounds
+    # the paper's network sizes (Sec. 5): n = 130 (32-column tiles) and n = 1026 (8-column tiles, eleven rounds)
+    "consensus_fused_130": dict(kind="consensus", n=130, d=1 << 20, variant=2, fused=1),
     "consensus_fused_1026": dict(kind="consensus", n=1026, d=1 << 18, variant=2, fused=1),
     "consensus_rounds_1026": dict(kind="consensus", n=1026, d=1 << 18, variant=2, fused=0),
     "logreg_grad": dict(kind="logreg", n=63, m=2000, d=4096, variant=2, gamma=0.01),
@@ -59,17 +63,34 @@ WORKLOADS = {
 }
 
 FALLBACK_HBM_GBS = 6650.0
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
-# capture summarised under profiles/ (None until captured, or once the kernel has changed since).
-NCU_TRAFFIC_BYTES_PER_LAUNCH = {
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, each from one ncu
+# capture: (bytes per launch, summary under profiles/, source file of the kernel, sha256 prefix of that
+# file when the counters were taken).  A kernel source that has changed since makes the entry stale
+# and `traffic` is reported as null until the capture is redone.
+NCU_TRAFFIC = {
     # 19.76 B per agent-parameter measured on step_small (2.5166 GB read + 1.6263 GB written for
-    # 100 x 2,097,152 units); traffic is proportional to the units, scaled here to n*d of each workload
-    "step_small": 4.143e9,
-    "resnet50_step": 19.755 * 100 * 25_557_032,
-    "consensus_fused": 1.165e9,
-    "consensus_rounds": 10.56e9,
-    "logreg_grad": 2.0736e9 + 29.9e6,
+    # 100 x 2,097,152 units); traffic is proportional to the units, scaled to n*d of resnet50_step
+    "step_small": (4.143e9, "step_walk_kernel__step_small__ncu_full.md", "step.cu", "955600f7f709"),
+    "resnet50_step": (19.755 * 100 * 25_557_032, "step_walk_kernel__step_small__ncu_full.md", "step.cu", "955600f7f709"),
+    "consensus_rounds": (10.56e9, "step_walk_kernel__consensus_rounds_n97_d1M__dram.md", "step.cu", "955600f7f709"),
+    "logreg_grad": (2.0736e9 + 29.9e6, "logreg_fused_kernel__n63_m2000_d4096__ncu_full.md", "logreg.cu", "e8cef610359e"),
 }
+
+
+def ncu_traffic(workload):
+    """Bytes per launch from the recorded capture, or None when there is none or the kernel has changed."""
+    import hashlib
+    entry = NCU_TRAFFIC.get(workload)
+    if entry is None:
+        return None
+    value, _summary, source, digest = entry
+    path = os.path.join(ROOT, "paper_2306_00256_b200", "csrc", source)
+    try:
+        with open(path, "rb") as f:
+            current = hashlib.sha256(f.read()).hexdigest()
+    except OSError:
+        return None
+    return value if current.startswith(digest) else None
 
 
 def measured_peak():
@@ -262,7 +283,7 @@ def bench_step(args, wl, device, dist):
         peak, which = measured_peak()
         achieved = (12 * n * d if x_only else algorithmic_bytes_step(n, d, True)) / (avg_ms * 1e-3) / 1e9
         roof = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH.get(args.workload),
+                "traffic": ncu_traffic(args.workload),
                 "kernel": "step_walk_kernel<float4, gradient, %s>" % ("X only" if x_only else "reads Y"), "peak_source": "of " + which,
                 "avg_launch_ms": avg_ms, "median_launch_ms": statistics.median(dominant), "best_launch_ms": min(dominant),
                 "launches_timed": len(dominant),
@@ -323,6 +344,8 @@ def bench_step_e2e(args, wl, device):
 
 
 def bench_consensus(args, wl, device, dist):
+    """tau aligned rounds per step (one fused launch, or tau per-round launches); every step has its own
+    CUDA-event pair, and the host time of the call (argument checks, schedule, launch) is taken beside it."""
     import torch
     import paper_2306_00256_b200 as ceca
     import synthetic_inputs as synth
@@ -336,23 +359,36 @@ def bench_consensus(args, wl, device, dist):
         ceca.ceca_consensus_rounds(X, None, variant, 0, tau, fused, X_out=Xo, Y_out=Yo, workspace=ws)
     sampler = ClockSampler(torch.cuda.current_device())
     sampler.start()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
+    host_us = []
     torch.cuda.synchronize()
-    e0.record(stream)
-    for _ in range(args.steps):
+    ev[0].record(stream)
+    for s in range(args.steps):
+        t0 = time.perf_counter()
         ceca.ceca_consensus_rounds(X, None, variant, 0, tau, fused, X_out=Xo, Y_out=Yo, workspace=ws)
-    e1.record(stream)
+        host_us.append((time.perf_counter() - t0) * 1e6)
+        ev[s + 1].record(stream)
     torch.cuda.synchronize()
     clocks = sampler.stop()
-    total_ms = e0.elapsed_time(e1)
+    total_ms = ev[0].elapsed_time(ev[-1])
+    per_call = [ev[s].elapsed_time(ev[s + 1]) for s in range(args.steps)]
     assert ceca.ceca_read_status(ws) == 0
     peak, which = measured_peak()
     per_elem = 12 if fused else (16 * tau - 4)   # fused: X in, X and Y out; per round: 16 B (12 B in round 0)
-    achieved = per_elem * n * d / (total_ms / args.steps * 1e-3) / 1e9
+    avg_ms = total_ms / args.steps
+    achieved = per_elem * n * d / (avg_ms * 1e-3) / 1e9
+    if not fused:
+        kernel = "step_walk_kernel<float4, no gradient> x tau"
+    elif fused == 3:
+        kernel = "consensus_tmem_kernel (tensor-memory exchange)"
+    elif fused == 2 or n > 256 or variant != 2:
+        kernel = "consensus_fused_kernel (shared-memory exchange of every row)"
+    else:
+        kernel = "consensus_block_kernel (register blocks, boundary rows through shared memory)"
     roof = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-            "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH.get(args.workload),
-            "kernel": "consensus_fused_kernel" if fused else "step_walk_kernel<float4, no gradient> x tau",
-            "peak_source": "of " + which}
+            "traffic": ncu_traffic(args.workload), "kernel": kernel, "peak_source": "of " + which,
+            "avg_launch_ms": avg_ms, "median_launch_ms": statistics.median(per_call), "best_launch_ms": min(per_call),
+            "host_us_per_call": round(statistics.median(host_us), 1)}
     launches = args.steps * (1 if fused else tau)
     return total_ms, launches, roof, clocks, {"tau": tau, "rounds_per_step": tau,
                                                "l2": "X is %d MB, larger than L2; outputs go to separate buffers" % (n * d * 4 // 1000000)}
@@ -390,7 +426,7 @@ def bench_logreg(args, wl, device, dist):
     peak, which = measured_peak()
     achieved = (4 * n * m * d + 8 * n * d + 4 * n * m) / (grad_ms * 1e-3) / 1e9
     roof = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-            "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH.get(args.workload),
+            "traffic": ncu_traffic(args.workload),
             "kernel": "logreg_fused_kernel + logreg_reduce_kernel", "peak_source": "of " + which, "avg_launch_ms": grad_ms}
     return total_ms, 3 * args.steps, roof, clocks, {"m": m, "l2": "A is 2.06 GB, larger than L2"}
 

@@ -12,7 +12,11 @@
  *     is an even row.
  *   - Pointers named X, Y, G, A, labels, *_out and workspace are DEVICE pointers unless the
  *     function name ends in _host.  The caller owns every buffer; the library allocates no
- *     device memory, keeps no global state between calls and never frees anything.
+ *     device memory and never frees anything.  What it keeps between calls is small and holds no
+ *     problem data: per-device constants (SM count, kernel attributes set once) and a cache of
+ *     encoded TMA tensor maps keyed on (pointer, n, d, ld).  Two entry points go further and say
+ *     so below: dsgd_logreg_grad_static (a fixed scratch buffer inside the library) and
+ *     ceca_gossip_sgd_step_host (internal streams, created and destroyed per call).
  *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
  *     Device entry points only enqueue work: they do not synchronise and return as soon
  *     as the launches are queued.
@@ -40,7 +44,7 @@ typedef enum {
   CECA_ERR_INVALID_ARG = 1, /* NULL where data is needed, n < 1, d < 1, ld < d, k < 0, ...       */
   CECA_ERR_ODD_N_1P = 2,    /* CECA-1P is defined for even n only (Sec. 3.2)                     */
   CECA_ERR_ALIGNMENT = 3,   /* the fused consensus kernel needs 16-byte aligned rows             */
-  CECA_ERR_UNSUPPORTED = 4, /* e.g. crossed aliasing of X/Y buffers, fused path with n > 2048      */
+  CECA_ERR_UNSUPPORTED = 4, /* e.g. crossed aliasing of X/Y buffers, a fused kernel outside its range of n */
   CECA_ERR_WORKSPACE = 5,   /* workspace NULL or smaller than ceca_workspace_bytes says          */
   CECA_ERR_CUDA = 6,        /* a CUDA runtime / driver call failed (launch, copy, map encode)    */
   CECA_ERR_STATIC_SCRATCH = 7 /* dsgd_logreg_grad_static: the problem needs more scratch than the
@@ -111,19 +115,28 @@ ceca_status_t ceca_gossip_sgd_step(const float *X, const float *Y, const float *
  *   fused = 0: one kernel launch per round, each a full pass over HBM.  Works for every n, d,
  *              ld and alignment.  Y_out == NULL is allowed when workspace holds n*ld floats, and
  *              without any workspace when n is a power of two (J then never feeds I).
- *   fused = 1: a single launch.  A column tile of all n rows is brought into shared memory by
- *              TMA (cp.async.bulk.tensor), every round runs on chip, and the tile is written
- *              back once.  Needs n <= 2048 (32-column tiles up to n = 256, 8-column tiles above),
- *              X / X_out (and Y / Y_out when used) 16-byte aligned
- *              with ld*4 a multiple of 16 (else CECA_ERR_ALIGNMENT), ld < 2^32 (more than 64 rounds
- *              run as several launches and then need Y_out),
- *              and a workspace of ceca_workspace_bytes(CECA_WS_CONSENSUS_FUSED, ...) bytes
+ *   fused = 1 (CECA_FUSED_AUTO): a single launch.  A column tile of all n rows is brought on chip
+ *              by TMA (cp.async.bulk.tensor), every round runs there, and the tile is written back
+ *              once.  Two kernels exist and 1 picks by n:
+ *                2 (CECA_FUSED_SMEM) exchanges the rows through shared memory; n <= 2048 (32-column
+ *                  tiles up to n = 256, 8-column tiles above);
+ *                3 (CECA_FUSED_TMEM) exchanges them through tensor memory (tcgen05.st / tcgen05.ld)
+ *                  and is the faster one where it applies: 2 <= n <= 128.
+ *              Passing 2 or 3 forces that kernel (CECA_ERR_UNSUPPORTED outside its range).
+ *              All need X / X_out (and Y / Y_out when used) 16-byte aligned with ld*4 a multiple of
+ *              16 (else CECA_ERR_ALIGNMENT), ld < 2^32 (more than 64 rounds run as several
+ *              launches and then need Y_out), and a workspace of
+ *              ceca_workspace_bytes(CECA_WS_CONSENSUS_FUSED, ...) bytes
  *              whose first int32 is a status word: it is left unchanged when the launch
  *              completes normally and set non-zero if a bounded on-chip wait for a TMA
- *              transfer ran out (read it with ceca_read_status).  Y may be NULL when the
- *              first round is r = 0; Y_out may be NULL.
- * X_out == X (and Y_out == Y) in place is allowed in both modes.
+ *              transfer ran out (read it with ceca_read_status); the tiles concerned are then
+ *              not written.  Y may be NULL when the first round is r = 0; Y_out may be NULL.
+ * X_out == X (and Y_out == Y) in place is allowed in every mode.
  */
+typedef enum {
+  CECA_UNFUSED = 0, CECA_FUSED_AUTO = 1, CECA_FUSED_SMEM = 2, CECA_FUSED_TMEM = 3, CECA_FUSED_BLOCK = 4
+} ceca_fused_t;
+
 ceca_status_t ceca_consensus_rounds(const float *X, const float *Y, float *X_out, float *Y_out,
                                     int32_t n, int64_t d, int64_t ld, ceca_variant_t variant,
                                     int64_t k0, int32_t rounds, int32_t fused, void *workspace,
@@ -203,6 +216,19 @@ size_t ceca_workspace_bytes(ceca_workspace_kind_t kind, int32_t n, int32_t m, in
  * (cudaMemsetAsync) before the first launch that uses the workspace.
  */
 ceca_status_t ceca_read_status(const void *workspace, int32_t *status_out, void *stream);
+
+/*
+ * Self-test of the bounded on-chip wait (no counterpart in the paper; meant for test suites, not for
+ * production calls).  Launches the fused consensus kernel named by `fused` (CECA_FUSED_SMEM or
+ * CECA_FUSED_TMEM) for one CECA-2P round on X, with the barrier that guards the TMA landing armed for
+ * 16 bytes more than the transfer delivers and a poll budget of a few thousand polls.  The
+ * transfer itself completes normally and nothing stays in flight; only the wait cannot succeed, so
+ * every tile gives up: the status word at the start of `workspace` becomes non-zero and X_out
+ * (which must not alias X) is left untouched.  Nothing traps; the context stays usable, and after
+ * the word is cleared an ordinary call works as before.  Arguments as for ceca_consensus_rounds.
+ */
+ceca_status_t ceca_fused_wait_selftest(const float *X, float *X_out, int32_t n, int64_t d, int64_t ld,
+                                       int32_t fused, void *workspace, size_t workspace_bytes, void *stream);
 
 /*
  * The same iteration as ceca_gossip_sgd_step for callers whose data lives in HOST memory

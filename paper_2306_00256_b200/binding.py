@@ -8,6 +8,7 @@ from . import build as _build
 
 CECA_1P = 1
 CECA_2P = 2
+UNFUSED, FUSED_AUTO, FUSED_SMEM, FUSED_TMEM, FUSED_BLOCK = 0, 1, 2, 3, 4
 WS_CONSENSUS_FUSED = 1
 WS_CONSENSUS_UNFUSED = 2
 WS_LOGREG_GRAD = 3
@@ -15,7 +16,8 @@ WS_STEP_HOST = 4
 
 EXPORTS = ["ceca_schedule", "ceca_gossip_sgd_step", "ceca_consensus_rounds", "dsgd_logreg_grad",
            "ceca_workspace_bytes", "ceca_read_status", "ceca_gossip_sgd_step_host", "ceca_status_string",
-           "dsgd_logreg_grad_static", "dsgd_logreg_grad_static_capacity", "dsgd_lsq_grad"]
+           "dsgd_logreg_grad_static", "dsgd_logreg_grad_static_capacity", "dsgd_lsq_grad",
+           "ceca_fused_wait_selftest"]
 
 
 class Round(ctypes.Structure):
@@ -66,6 +68,8 @@ def library():
     lib.dsgd_logreg_grad_static_capacity.restype = ctypes.c_size_t
     lib.ceca_workspace_bytes.argtypes = [ctypes.c_int, i32, i32, i64]
     lib.ceca_workspace_bytes.restype = ctypes.c_size_t
+    lib.ceca_fused_wait_selftest.argtypes = [vp, vp, i32, i64, i64, i32, vp, ctypes.c_size_t, vp]
+    lib.ceca_fused_wait_selftest.restype = ctypes.c_int
     lib.ceca_read_status.argtypes = [vp, ctypes.POINTER(i32), vp]
     lib.ceca_read_status.restype = ctypes.c_int
     lib.ceca_gossip_sgd_step_host.argtypes = [vp, vp, vp, i32, i64, i64, f32, i32, i64, vp, ctypes.c_size_t]
@@ -150,9 +154,20 @@ def ceca_consensus_rounds(X, Y, variant, k0, rounds, fused, X_out=None, Y_out=No
             raise ValueError("%s must have the shape and row stride of X" % name)
     ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
     st = library().ceca_consensus_rounds(_ptr(X), _ptr(Y), _ptr(X_out), _ptr(Y_out), n, d, ld, variant, k0,
-                                         rounds, int(bool(fused)), _ptr(workspace), ws_bytes, _stream(stream))
+                                         rounds, int(fused), _ptr(workspace), ws_bytes, _stream(stream))
     _check(st, "ceca_consensus_rounds")
     return X_out, Y_out
+
+
+def ceca_fused_wait_selftest(X, X_out, fused, workspace, stream=None):
+    """Runs the named fused consensus kernel with a landing barrier that cannot complete (test suites only)."""
+    n, d, ld = _matrix(X, "X")
+    if _matrix(X_out, "X_out", n) != (n, d, ld):
+        raise ValueError("X_out must have the shape and row stride of X")
+    ws_bytes = workspace.numel() * workspace.element_size()
+    st = library().ceca_fused_wait_selftest(_ptr(X), _ptr(X_out), n, d, ld, int(fused), _ptr(workspace), ws_bytes,
+                                            _stream(stream))
+    _check(st, "ceca_fused_wait_selftest")
 
 
 def dsgd_logreg_grad(A, labels, X, Y, k, variant, G, workspace, stream=None):

@@ -16,11 +16,13 @@
 #include <cuda.h>
 #include <cuda_runtime.h>
 
+#include <atomic>
 #include <cstdint>
 #include <cstring>
 
 #include "ceca.h"
 #include "plan.h"
+#include "tma.h"
 
 namespace ceca {
 
@@ -28,6 +30,14 @@ cudaError_t enqueue_step(const Plan &plan, const float *X, const float *Y, const
                          float *Yo, int32_t n, int64_t d, int64_t ld, float gamma,
                          cudaStream_t stream);
 ceca_status_t check_matrix_args(const void *X, const void *X_out, int32_t n, int64_t d, int64_t ld);
+bool consensus_block_supports(int32_t n, ceca_variant_t variant, int32_t rounds, bool y_in);
+ceca_status_t consensus_block(const float *X, const float *Y, float *Xo, float *Yo, int32_t n, int64_t d,
+                              int64_t ld, int64_t k0, int32_t rounds, int32_t *status, int32_t wait_polls,
+                              uint32_t tx_extra, cudaStream_t stream);
+bool consensus_tmem_supports(int32_t n, int32_t rounds);
+ceca_status_t consensus_tmem(const float *X, const float *Y, float *Xo, float *Yo, int32_t n, int64_t d,
+                             int64_t ld, ceca_variant_t variant, int64_t k0, int32_t rounds, int32_t *status,
+                             int32_t wait_polls, uint32_t tx_extra, cudaStream_t stream);
 
 constexpr int kMaxFusedRounds = 64;
 constexpr int kMaxBoxRows = 256;     // one TMA box holds at most 256 rows; taller tiles take several boxes
@@ -46,52 +56,11 @@ struct FusedRound {
 struct FusedArgs {
   int32_t n, rounds, one_port, has_y_in, has_y_out;
   int32_t boxes, box_rows;  // the tile is `boxes` TMA boxes of `box_rows` rows (boxes * box_rows >= n)
+  int32_t wait_polls;       // poll budget of the bounded wait for the tile
+  uint32_t tx_extra;        // added to the byte count the landing barrier is armed for (0 except in the self-test)
   int32_t *status;
   FusedRound rd[kMaxFusedRounds];
 };
-
-// ---- PTX wrappers (mbarrier + TMA) ----------------------------------------------------------
-__device__ __forceinline__ uint32_t smem_u32(const void *p) {
-  return (uint32_t)__cvta_generic_to_shared(p);
-}
-__device__ __forceinline__ void mbar_init(uint64_t *bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
-}
-__device__ __forceinline__ void mbar_expect_tx(uint64_t *bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes)
-               : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t phase) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok)
-      : "r"(smem_u32(bar)), "r"(phase)
-      : "memory");
-  return ok != 0;
-}
-// Bounded wait: returns false when the barrier did not flip within the poll budget.
-__device__ __forceinline__ bool mbar_wait_bounded(uint64_t *bar, uint32_t phase, uint32_t polls) {
-  for (uint32_t i = 0; i < polls; ++i) {
-    if (mbar_try_wait(bar, phase)) return true;
-    __nanosleep(64);
-  }
-  return false;
-}
-__device__ __forceinline__ void tma_load_2d(void *dst, const CUtensorMap *map, int32_t x, int32_t y,
-                                            uint64_t *bar) {
-  asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-      ::"r"(smem_u32(dst)), "l"(map), "r"(x), "r"(y), "r"(smem_u32(bar))
-      : "memory");
-}
-__device__ __forceinline__ void tma_store_2d(const CUtensorMap *map, int32_t x, int32_t y, const void *src) {
-  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];"
-               ::"l"(map), "r"(x), "r"(y), "r"(smem_u32(src))
-               : "memory");
-}
 
 __device__ __forceinline__ float4 mix4(float w_own, float4 own, float w_recv, float4 recv) {
   // w_own * own + w_recv * recv on four lanes with two-wide packed fp32 instructions
@@ -134,24 +103,24 @@ consensus_fused_kernel(const __grid_constant__ CUtensorMap map_x_in, const __gri
 
   if (threadIdx.x == 0) {
     mbar_init(&bar, 1);
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    mbar_fence_init();
   }
   __syncthreads();
   if (threadIdx.x == 0) {
     const uint32_t tile_bytes = (uint32_t)tile_rows * kTileCols * sizeof(float);  // boxes count in full
-    mbar_expect_tx(&bar, p.has_y_in ? 2 * tile_bytes : tile_bytes);
+    mbar_expect_tx(&bar, (p.has_y_in ? 2 * tile_bytes : tile_bytes) + p.tx_extra);
     for (int b = 0; b < p.boxes; ++b) {  // rows past n are out of range for the tensor map: zero fill
       const int row0 = b * p.box_rows;
       tma_load_2d(tile_a + (size_t)row0 * kTileCols, &map_x_in, col0, row0, &bar);
       if (p.has_y_in) tma_load_2d(tile_b + (size_t)row0 * kTileCols, &map_y_in, col0, row0, &bar);
     }
   }
-  const bool landed = mbar_wait_bounded(&bar, 0, kWaitPolls);
+  const bool landed = mbar_wait_bounded(&bar, 0, (uint32_t)p.wait_polls);
   if (!__syncthreads_and(landed)) {  // one decision for the whole CTA
     // The transfer never arrived: flag it, give it one more bounded chance to land (so that
     // it cannot write into shared memory of a finished CTA), and give up without storing.
     if (threadIdx.x == 0) atomicExch(p.status, 1);
-    mbar_wait_bounded(&bar, 0, kWaitPolls);
+    mbar_wait_bounded(&bar, 0, (uint32_t)p.wait_polls);
     return;
   }
 
@@ -247,46 +216,15 @@ consensus_fused_kernel(const __grid_constant__ CUtensorMap map_x_in, const __gri
 }
 
 // ---- host side ------------------------------------------------------------------------------
-typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
-                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *,
-                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
-                                  CUtensorMapFloatOOBfill);
-
-static EncodeTiledFn encode_tiled_fn() {
-  static EncodeTiledFn fn = []() -> EncodeTiledFn {
-    void *sym = nullptr;
-    cudaDriverEntryPointQueryResult q;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &q) != cudaSuccess ||
-        q != cudaDriverEntryPointSuccess)
-      return nullptr;
-    return reinterpret_cast<EncodeTiledFn>(sym);
-  }();
-  return fn;
-}
-
-// An n x d fp32 matrix with row pitch ld, boxed as box_rows rows x tile_cols columns.
-static bool make_map(CUtensorMap *map, const float *base, int32_t n, int64_t d, int64_t ld, int tile_cols,
-                     int box_rows) {
-  EncodeTiledFn enc = encode_tiled_fn();
-  if (!enc) return false;
-  const cuuint64_t dims[2] = {(cuuint64_t)d, (cuuint64_t)n};
-  const cuuint64_t strides[1] = {(cuuint64_t)ld * sizeof(float)};
-  const cuuint32_t box[2] = {(cuuint32_t)tile_cols, (cuuint32_t)box_rows};
-  const cuuint32_t elem[2] = {1, 1};
-  return enc(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float *>(base), dims, strides, box, elem,
-             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
 template <int R, int W, int T>
 static cudaError_t launch_fused(const CUtensorMap &mxi, const CUtensorMap &myi, const CUtensorMap &mxo,
                                 const CUtensorMap &myo, const FusedArgs &args, int64_t d, cudaStream_t stream) {
   const size_t smem = 2 * (size_t)args.boxes * args.box_rows * W * sizeof(float);
-  cudaError_t e = cudaFuncSetAttribute(consensus_fused_kernel<R, W, T>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       (int)smem);
-  if (e != cudaSuccess) return e;
-  e = cudaFuncSetAttribute(consensus_fused_kernel<R, W, T>, cudaFuncAttributePreferredSharedMemoryCarveout,
-                           cudaSharedmemCarveoutMaxShared);
+  // the largest tile this instantiation is ever launched with: R rows for each of its row groups
+  constexpr size_t kMaxSmem = 2 * (size_t)R * (T / (W / 8)) * W * sizeof(float);
+  static std::atomic<uint64_t> attr_done{0};
+  cudaError_t e = set_max_shared_once(reinterpret_cast<const void *>(consensus_fused_kernel<R, W, T>),
+                                      kMaxSmem < smem ? smem : kMaxSmem, &attr_done);
   if (e != cudaSuccess) return e;
   const int64_t tiles = (d + W - 1) / W;
   consensus_fused_kernel<R, W, T><<<(unsigned)tiles, T, smem, stream>>>(mxi, myi, mxo, myo, args);
@@ -295,16 +233,23 @@ static cudaError_t launch_fused(const CUtensorMap &mxi, const CUtensorMap &myi, 
 
 static inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
+// `kind`: a ceca_fused_t other than CECA_UNFUSED.
+// wait_polls <= 0: the default poll budget; tx_extra: see FusedArgs (self-test only).
 static ceca_status_t consensus_fused(const float *X, const float *Y, float *Xo, float *Yo, int32_t n, int64_t d,
-                                     int64_t ld, ceca_variant_t variant, int64_t k0, int32_t rounds,
-                                     void *workspace, size_t workspace_bytes, cudaStream_t stream) {
+                                     int64_t ld, ceca_variant_t variant, int64_t k0, int32_t rounds, int kind,
+                                     void *workspace, size_t workspace_bytes, int32_t wait_polls, uint32_t tx_extra,
+                                     cudaStream_t stream) {
   if (n > kMaxFusedRows || rounds > kMaxFusedRounds || ld >= ((int64_t)1 << 32) || d > 0x7fffffffLL)
     return CECA_ERR_UNSUPPORTED;
+  if (kind == CECA_FUSED_TMEM && !consensus_tmem_supports(n, rounds)) return CECA_ERR_UNSUPPORTED;
+
   if (!workspace || workspace_bytes < sizeof(int32_t) || !aligned16(workspace)) return CECA_ERR_WORKSPACE;
   FusedArgs args;
   std::memset(&args, 0, sizeof(args));
   args.n = n; args.rounds = rounds; args.one_port = (variant == CECA_1P);
   args.status = static_cast<int32_t *>(workspace);
+  args.wait_polls = wait_polls > 0 ? wait_polls : (int32_t)kWaitPolls;
+  args.tx_extra = tx_extra;
   bool first_needs_y = false;
   for (int32_t t = 0; t < rounds; ++t) {
     Plan plan;
@@ -323,6 +268,15 @@ static ceca_status_t consensus_fused(const float *X, const float *Y, float *Xo, 
       (Yo && !aligned16(Yo)))
     return CECA_ERR_ALIGNMENT;
 
+  const bool block_ok = consensus_block_supports(n, variant, rounds, args.has_y_in != 0);
+  if (kind == CECA_FUSED_BLOCK && !block_ok) return CECA_ERR_UNSUPPORTED;
+  if (kind == CECA_FUSED_BLOCK || (kind == CECA_FUSED_AUTO && block_ok))
+    return consensus_block(X, args.has_y_in ? Y : nullptr, Xo, Yo, n, d, ld, k0, rounds, args.status, wait_polls,
+                           tx_extra, stream);
+  if (kind == CECA_FUSED_TMEM)
+    return consensus_tmem(X, args.has_y_in ? Y : nullptr, Xo, Yo, n, d, ld, variant, k0, rounds, args.status,
+                          wait_polls, tx_extra, stream);
+
   // tile geometry: all n rows, 32 columns wide while one TMA box (256 rows) holds them, else 8
   const int tile_cols = n <= kMaxBoxRows ? kWideTileCols : kNarrowTileCols;
   args.boxes = (n + kMaxBoxRows - 1) / kMaxBoxRows;
@@ -330,10 +284,10 @@ static ceca_status_t consensus_fused(const float *X, const float *Y, float *Xo, 
   if (tile_cols == kNarrowTileCols)  // every box must start on a 128-byte boundary of shared memory
     args.box_rows = (args.box_rows + 3) / 4 * 4;
   CUtensorMap mxi, myi, mxo, myo;
-  if (!make_map(&mxi, X, n, d, ld, tile_cols, args.box_rows) || !make_map(&mxo, Xo, n, d, ld, tile_cols, args.box_rows))
+  if (!tensor_map_2d(&mxi, X, n, d, ld, tile_cols, args.box_rows) || !tensor_map_2d(&mxo, Xo, n, d, ld, tile_cols, args.box_rows))
     return CECA_ERR_CUDA;
-  if (!make_map(&myi, args.has_y_in ? Y : X, n, d, ld, tile_cols, args.box_rows)) return CECA_ERR_CUDA;
-  if (!make_map(&myo, Yo ? Yo : Xo, n, d, ld, tile_cols, args.box_rows)) return CECA_ERR_CUDA;
+  if (!tensor_map_2d(&myi, args.has_y_in ? Y : X, n, d, ld, tile_cols, args.box_rows)) return CECA_ERR_CUDA;
+  if (!tensor_map_2d(&myo, Yo ? Yo : Xo, n, d, ld, tile_cols, args.box_rows)) return CECA_ERR_CUDA;
 
   cudaError_t e;
   if (tile_cols == kWideTileCols) {
@@ -370,7 +324,9 @@ extern "C" ceca_status_t ceca_consensus_rounds(const float *X, const float *Y, f
   if (st != CECA_OK) return st;
   cudaStream_t stream = static_cast<cudaStream_t>(stream_);
 
+  if (fused < 0 || fused > CECA_FUSED_BLOCK) return CECA_ERR_INVALID_ARG;
   if (rounds == 0 || n == 1) {  // nothing to mix: the result is a copy of the input
+    if (Y_out && !Y) return CECA_ERR_INVALID_ARG;
     cudaError_t e = cudaSuccess;
     if (X_out != X)
       e = cudaMemcpy2DAsync(X_out, ld * sizeof(float), X, ld * sizeof(float), d * sizeof(float), n,
@@ -378,7 +334,6 @@ extern "C" ceca_status_t ceca_consensus_rounds(const float *X, const float *Y, f
     if (e == cudaSuccess && Y_out && Y && Y_out != Y)
       e = cudaMemcpy2DAsync(Y_out, ld * sizeof(float), Y, ld * sizeof(float), d * sizeof(float), n,
                             cudaMemcpyDeviceToDevice, stream);
-    if (Y_out && !Y) return CECA_ERR_INVALID_ARG;
     return e == cudaSuccess ? CECA_OK : CECA_ERR_CUDA;
   }
 
@@ -389,8 +344,8 @@ extern "C" ceca_status_t ceca_consensus_rounds(const float *X, const float *Y, f
     const float *x_in = X, *y_in = Y;
     for (int32_t done = 0; done < rounds; done += kMaxFusedRounds) {
       const int32_t chunk = rounds - done < kMaxFusedRounds ? rounds - done : kMaxFusedRounds;
-      st = consensus_fused(x_in, y_in, X_out, Y_out, n, d, ld, variant, k0 + done, chunk, workspace,
-                           workspace_bytes, stream);
+      st = consensus_fused(x_in, y_in, X_out, Y_out, n, d, ld, variant, k0 + done, chunk, fused, workspace,
+                           workspace_bytes, 0, 0, stream);
       if (st != CECA_OK) return st;
       x_in = X_out; y_in = Y_out;
     }
@@ -428,6 +383,21 @@ extern "C" ceca_status_t ceca_consensus_rounds(const float *X, const float *Y, f
     x_in = X_out; y_in = y_work;  // later rounds run in place on the outputs
   }
   return CECA_OK;
+}
+
+extern "C" ceca_status_t ceca_fused_wait_selftest(const float *X, float *X_out, int32_t n, int64_t d, int64_t ld,
+                                                  int32_t fused, void *workspace, size_t workspace_bytes,
+                                                  void *stream) {
+  using namespace ceca;
+  ceca_status_t st = check_matrix_args(X, X_out, n, d, ld);
+  if (st != CECA_OK) return st;
+  if (fused != CECA_FUSED_SMEM && fused != CECA_FUSED_TMEM && fused != CECA_FUSED_BLOCK) return CECA_ERR_INVALID_ARG;
+  if ((const float *)X_out == X || n < 2) return CECA_ERR_UNSUPPORTED;
+  // One round of CECA-2P from k0 = 0, with the landing barrier armed for 16 bytes more than the
+  // tile delivers and a poll budget of a few thousand: the transfer itself completes normally,
+  // only the wait cannot succeed.
+  return consensus_fused(X, nullptr, X_out, nullptr, n, d, ld, CECA_2P, 0, 1, fused, workspace, workspace_bytes,
+                         /*wait_polls=*/2048, /*tx_extra=*/16, static_cast<cudaStream_t>(stream));
 }
 
 extern "C" ceca_status_t ceca_read_status(const void *workspace, int32_t *status_out, void *stream) {

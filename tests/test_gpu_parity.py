@@ -260,18 +260,41 @@ def _fused_ws():
     return torch.zeros(64, dtype=torch.int32, device=DEV)
 
 
-@pytest.mark.parametrize("fused", [0, 1])
-@pytest.mark.parametrize("n", [2, 5, 6, 24, 63, 97, 100, 128, 130, 200, 256])
+def _fused_kernels(n, variant=ceca.CECA_2P):
+    """The fused kernels that take n agents and this variant: shared-memory exchange (n <= 2048),
+    tensor-memory exchange (n <= 128), register blocks (CECA-2P, n <= 256)."""
+    kernels = [ceca.FUSED_SMEM]
+    if n <= 128:
+        kernels.append(ceca.FUSED_TMEM)
+    if n <= 226 and variant == ceca.CECA_2P:   # (up to 256 when the first round does not read Y)
+        kernels.append(ceca.FUSED_BLOCK)
+    return kernels
+
+
+@pytest.mark.parametrize("fused", [ceca.UNFUSED, ceca.FUSED_SMEM, ceca.FUSED_TMEM, ceca.FUSED_BLOCK])
+@pytest.mark.parametrize("n", [2, 3, 4, 5, 6, 7, 8, 9, 16, 17, 24, 31, 33, 63, 65, 97, 100, 127, 128, 129, 130, 200, 255, 256])
 @pytest.mark.parametrize("d", [32, 1000, 4100])
 def test_consensus_matches_oracle_and_reaches_the_mean(fused, n, d):
+    if fused == ceca.FUSED_TMEM and n > 128:
+        with pytest.raises(ceca.CecaError):   # outside that kernel's range: refused, nothing launched
+            ceca.ceca_consensus_rounds(torch.zeros(n, d, device=DEV), None, ceca.CECA_2P, 0, 1, fused, workspace=_fused_ws(),
+                                       want_y=False)
+        return
     x = synth.consensus_inputs(n, d, seed=n + d)
     y0 = synth.consensus_inputs(n, d, seed=n + d + 1, offset_rows=False)
     tau = _tau(n)
     for variant in _variants(n):
+        if fused == ceca.FUSED_BLOCK and variant != ceca.CECA_2P:
+            continue
         for k0, rounds in [(0, tau), (0, tau + 1), (0, 1), (1 % tau, 2 * tau + 3), (5 * tau, tau)]:
             X, Y = x.to(DEV), y0.to(DEV)
             Xo, Yo = torch.empty_like(X), torch.empty_like(Y)
             ws = _fused_ws()
+            if fused == ceca.FUSED_BLOCK and n > 226 and k0 % tau:
+                # a first round that reads Y needs a fourth shared-memory tile, which no longer fits
+                with pytest.raises(ceca.CecaError):
+                    ceca.ceca_consensus_rounds(X, Y, variant, k0, rounds, fused, X_out=Xo, Y_out=Yo, workspace=ws)
+                continue
             ceca.ceca_consensus_rounds(X, Y, variant, k0, rounds, fused, X_out=Xo, Y_out=Yo, workspace=ws)
             assert ceca.ceca_read_status(ws) == 0
             want_x, want_y = oracle.consensus(_np(x), _np(y0), variant, k0, rounds)
@@ -344,17 +367,18 @@ def test_finite_time_consensus_for_every_network_size():
         assert tau == int(np.ceil(np.log2(n)))
         for variant in _variants(n):
             ws = _fused_ws()
-            for rounds, reached in ((tau - 1, False), (tau, True)):
-                if rounds == 0:
-                    continue
-                Xo, Yo = torch.empty(n, d, device=DEV), torch.empty(n, d, device=DEV)
-                ceca.ceca_consensus_rounds(x.to(DEV), y.to(DEV), variant, 0, rounds, 1, X_out=Xo, Y_out=Yo, workspace=ws)
-                residue = float((Xo.double().cpu() - mean).norm(dim=1).sum()) / n
-                assert (residue < 1e-5) == reached, (n, variant, rounds, residue)
+            for fused in _fused_kernels(n, variant):
+                for rounds, reached in ((tau - 1, False), (tau, True)):
+                    if rounds == 0:
+                        continue
+                    Xo, Yo = torch.empty(n, d, device=DEV), torch.empty(n, d, device=DEV)
+                    ceca.ceca_consensus_rounds(x.to(DEV), y.to(DEV), variant, 0, rounds, fused, X_out=Xo, Y_out=Yo, workspace=ws)
+                    residue = float((Xo.double().cpu() - mean).norm(dim=1).sum()) / n
+                    assert (residue < 1e-5) == reached, (n, variant, fused, rounds, residue)
             assert ceca.ceca_read_status(ws) == 0
 
 
-@pytest.mark.parametrize("fused", [0, 1])
+@pytest.mark.parametrize("fused", [0, 1, 2, 3, 4])
 def test_consensus_optional_y(fused):
     n, d = 97, 1000
     x = synth.consensus_inputs(n, d, seed=5)
@@ -385,34 +409,42 @@ def test_consensus_optional_y(fused):
     assert torch.equal(oc, one)
 
 
-def test_fused_consensus_many_rounds():
-    """More rounds than one launch takes: chunks of 64, continuing in place."""
+@pytest.mark.parametrize("fused", [ceca.FUSED_SMEM, ceca.FUSED_TMEM, ceca.FUSED_BLOCK])
+def test_fused_consensus_many_rounds(fused):
+    """More rounds than one launch takes: chunks of 64, continuing in place (the tensor-memory kernel
+    also folds its running scales back every 16 rounds)."""
     n, d, rounds, k0 = 12, 200, 150, 5
     x = synth.consensus_inputs(n, d, seed=3)
     y = synth.consensus_inputs(n, d, seed=4, offset_rows=False)
     for variant in (ceca.CECA_2P, ceca.CECA_1P):
+        if fused == ceca.FUSED_BLOCK and variant != ceca.CECA_2P:
+            continue
         Xo, Yo = torch.empty(n, d, device=DEV), torch.empty(n, d, device=DEV)
         ws = _fused_ws()
-        ceca.ceca_consensus_rounds(x.to(DEV), y.to(DEV), variant, k0, rounds, 1, X_out=Xo, Y_out=Yo, workspace=ws)
+        ceca.ceca_consensus_rounds(x.to(DEV), y.to(DEV), variant, k0, rounds, fused, X_out=Xo, Y_out=Yo, workspace=ws)
         assert ceca.ceca_read_status(ws) == 0
         want_x, want_y = oracle.consensus(_np(x), _np(y), variant, k0, rounds)
         tol = STEP_TOL * rounds * _scale(0, (x, 1), (y, 1))
         assert np.abs(_np(Xo) - want_x).max() <= tol and np.abs(_np(Yo) - want_y).max() <= tol
         with pytest.raises(ceca.CecaError):   # nowhere to keep Y between the launches
-            ceca.ceca_consensus_rounds(x.to(DEV), y.to(DEV), variant, k0, rounds, 1, X_out=Xo, workspace=ws, want_y=False)
+            ceca.ceca_consensus_rounds(x.to(DEV), y.to(DEV), variant, k0, rounds, fused, X_out=Xo, workspace=ws, want_y=False)
 
 
-def test_fused_consensus_padded_rows():
+@pytest.mark.parametrize("fused", [ceca.FUSED_SMEM, ceca.FUSED_TMEM, ceca.FUSED_BLOCK])
+def test_fused_consensus_padded_rows(fused):
     n, d, ld = 100, 1000, 1024
     x = synth.consensus_inputs(n, d, seed=9)
     (X, xb), (Xo, xob), (Yo, yob) = _put(x.to(DEV), ld), _padded(n, d, ld), _padded(n, d, ld)
     ws = _fused_ws()
     for variant in (ceca.CECA_2P, ceca.CECA_1P):
-        ceca.ceca_consensus_rounds(X, None, variant, 0, 7, 1, X_out=Xo, Y_out=Yo, workspace=ws)
+        if fused == ceca.FUSED_BLOCK and variant != ceca.CECA_2P:
+            continue
+        ceca.ceca_consensus_rounds(X, None, variant, 0, 7, fused, X_out=Xo, Y_out=Yo, workspace=ws)
         want_x, want_y = oracle.consensus(_np(x), np.zeros((n, d)), variant, 0, 7)
         tol = STEP_TOL * 7 * float(x.abs().max())
         assert np.abs(_np(Xo) - want_x).max() <= tol and np.abs(_np(Yo) - want_y).max() <= tol
-        assert torch.isnan(xob[:n * ld].view(n, ld)[:, d:]).all()   # TMA stores clip at column d
+        assert torch.isnan(xob[:n * ld].view(n, ld)[:, d:]).all()   # stores stop at column d
+        assert torch.isnan(yob[:n * ld].view(n, ld)[:, d:]).all()
         assert ceca.ceca_read_status(ws) == 0
 
 
@@ -447,7 +479,7 @@ def test_step_and_consensus_on_random_shapes():
         k0 = int(rng.integers(0, 40))
         ld4 = (d + 3) // 4 * 4 + 4 * int(rng.integers(0, 3))
         (Xc, _), (Yc, _) = _put(x.to(DEV), ld4, 0), _put(y.to(DEV), ld4, 0)
-        fused = int(n <= 2048 and rng.integers(0, 2))
+        fused = int(rng.choice([0, 1] + _fused_kernels(n, variant)))
         ws = _fused_ws()
         ceca.ceca_consensus_rounds(Xc, Yc, variant, k0, rounds, fused, workspace=ws)
         assert ceca.ceca_read_status(ws) == 0
@@ -455,6 +487,33 @@ def test_step_and_consensus_on_random_shapes():
         tol = STEP_TOL * rounds * _scale(0, (x, 1), (y, 1))
         assert np.abs(_np(Xc) - want_x).max() <= tol, (case, n, d, ld4, variant, k0, rounds, fused)
         assert np.abs(_np(Yc) - want_y).max() <= tol, (case, n, d, ld4, variant, k0, rounds, fused)
+
+
+@pytest.mark.parametrize("fused", [ceca.FUSED_SMEM, ceca.FUSED_TMEM, ceca.FUSED_BLOCK])
+def test_bounded_wait_of_the_fused_kernels_runs_out_and_reports(fused):
+    """The only device-side wait in the library is the wait for the TMA landing.  The self-test entry arms
+    that barrier for more bytes than arrive: every tile must give up after its poll budget, set the status
+    word, store nothing, and leave the context usable for an ordinary call."""
+    n, d = 6, 32
+    x = synth.consensus_inputs(n, d, seed=11)
+    X = x.to(DEV)
+    Xo = torch.full_like(X, float("nan"))
+    ws = _fused_ws()
+    ceca.ceca_fused_wait_selftest(X, Xo, fused, ws)
+    assert ceca.ceca_read_status(ws) == 1
+    assert torch.isnan(Xo).all() and torch.equal(X.cpu(), x)
+    ws.zero_()
+    ceca.ceca_consensus_rounds(X, None, ceca.CECA_2P, 0, 3, fused, X_out=Xo, workspace=ws, want_y=False)
+    assert ceca.ceca_read_status(ws) == 0
+    want_x, _ = oracle.consensus(_np(x), np.zeros((n, d)), ceca.CECA_2P, 0, 3)
+    assert np.abs(_np(Xo) - want_x).max() <= STEP_TOL * 3 * float(x.abs().max())
+    # several tiles per group and a ragged last tile
+    n, d = 97, 4100
+    X = synth.consensus_inputs(n, d, seed=12).to(DEV)
+    Xo = torch.full_like(X, float("nan"))
+    ws.zero_()
+    ceca.ceca_fused_wait_selftest(X, Xo, fused, ws)
+    assert ceca.ceca_read_status(ws) == 1 and torch.isnan(Xo).all()
 
 
 # --------------------------------------------------------------------------------------------
