@@ -49,6 +49,8 @@ WORKLOADS = {
     "consensus_fused_smem": dict(kind="consensus", n=97, d=1 << 20, variant=2, fused=2),
     "consensus_fused_tmem": dict(kind="consensus", n=97, d=1 << 20, variant=2, fused=3),
     "consensus_rounds": dict(kind="consensus", n=97, d=1 << 20, variant=2, fused=0),
+    # half the columns: the case the profiler captures are taken on (0.2 GB in, 0.4 GB out)
+    "consensus_fused_small": dict(kind="consensus", n=97, d=1 << 19, variant=2, fused=1),
     # the paper's network sizes (Sec. 5): n = 130 (32-column tiles) and n = 1026 (8-column tiles, eleven rounds)
     "consensus_fused_130": dict(kind="consensus", n=130, d=1 << 20, variant=2, fused=1),
     "consensus_fused_1026": dict(kind="consensus", n=1026, d=1 << 18, variant=2, fused=1),

@@ -40,6 +40,8 @@
 #include <atomic>
 #include <cstdint>
 #include <cstring>
+#include <type_traits>
+#include <utility>
 
 #include "ceca.h"
 #include "plan.h"
@@ -50,14 +52,20 @@ namespace ceca {
 constexpr int kBkTileCols = 64;
 constexpr int kBkMaxRounds = 64;
 constexpr int kBkRenormEvery = 16;
-constexpr int kBkMaxCb = 16;
+constexpr int kBkMaxCb = 25;            // agents per block (100 state registers)
 constexpr uint32_t kBkWaitPolls = 1u << 22;
+
+constexpr int kBkPayloadJ = 1;  // the message is J (else I)
+constexpr int kBkClearJ = 2;    // b = 0: J+ is the received value
+constexpr int kBkRenorm = 4;    // fold the running scales back into the values first
 
 struct BlockRound {
   float cI, cJ;        // Ih += cI * z_src, Jh += cJ * z_src
-  float preI, preJ;    // when renorm: Ih *= preI, Jh *= preJ first
-  int16_t hop;         // the shift s of this round
-  uint8_t payload, jclear, renorm, partial;  // partial: s < smallest block, the in-register form applies
+  float preI, preJ;    // with kBkRenorm: Ih *= preI, Jh *= preJ first
+  int32_t hop;         // the shift s of this round
+  int32_t mode;        // kBk* flags
+  int32_t sel;         // which instantiation of the round body runs (see dispatch_round)
+  int32_t pad;
 };
 
 struct BlockArgs {
@@ -65,6 +73,7 @@ struct BlockArgs {
   int64_t ld;
   int32_t d, n, rounds, has_y_in, has_y_out, tiles;
   int32_t nfull;       // blocks 0..nfull-1 hold CB agents, the others CB-1
+  int32_t single_xch;  // one exchange tile instead of two (saves shared memory, costs a second barrier per round)
   int32_t wait_polls;
   uint32_t tx_bytes;   // bytes the landing barrier is armed for
   float outI, outJ;
@@ -72,114 +81,183 @@ struct BlockArgs {
   BlockRound rd[kBkMaxRounds];
 };
 
-__device__ __forceinline__ float2 axpy2(float2 c, float2 z, float2 acc) { return __ffma2_rn(c, z, acc); }
+// Two adjacent columns travel as one 64-bit value (low word = the even column), so that the state
+// lives in aligned register pairs and the packed fp32 instructions take it without repacking.
+typedef unsigned long long pk2;
+__device__ __forceinline__ pk2 pk_make(float lo, float hi) {
+  pk2 v;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(v) : "f"(lo), "f"(hi));
+  return v;
+}
+__device__ __forceinline__ float pk_lo(pk2 v) { return __uint_as_float((unsigned)(v & 0xffffffffull)); }
+__device__ __forceinline__ pk2 axpy2(pk2 c, pk2 z, pk2 acc) {   // c * z + acc on both columns
+  pk2 d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(c), "l"(z), "l"(acc));
+  return d;
+}
+__device__ __forceinline__ pk2 mul2(pk2 c, pk2 v) {
+  pk2 d;
+  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(c), "l"(v));
+  return d;
+}
 
-// One round with a compile-time shift S smaller than every block.  `buf` is this round's exchange
-// tile, already offset to this thread's column pair; `full_block` says whether the block holds CB
-// rows (else CB-1).
+// Compile-time loop: f(integral_constant<int, 0>), ..., f(integral_constant<int, N-1>).
+template <int... Is, typename F>
+__device__ __forceinline__ void static_for_impl(std::integer_sequence<int, Is...>, F &&f) {
+  (f(std::integral_constant<int, Is>{}), ...);
+}
+template <int N, typename F>
+__device__ __forceinline__ void static_for(F &&f) {
+  static_for_impl(std::make_integer_sequence<int, N>{}, f);
+}
+#define CECA_IDX(I) decltype(I)::value
+
+// Shared memory is addressed by 32-bit shared-window addresses with compile-time byte offsets, so
+// that an access costs one instruction and no address arithmetic.
+constexpr int kBkRowBytes = kBkTileCols * (int)sizeof(float);
+template <int OFF>
+__device__ __forceinline__ pk2 lds64(uint32_t addr) {
+  pk2 v;
+  asm volatile("ld.shared.b64 %0, [%1+%2];" : "=l"(v) : "r"(addr), "n"(OFF) : "memory");
+  return v;
+}
+template <int OFF>
+__device__ __forceinline__ void sts64(uint32_t addr, pk2 v) {
+  asm volatile("st.shared.b64 [%0+%1], %2;" ::"r"(addr), "n"(OFF), "l"(v) : "memory");
+}
+
+// What a thread knows about its place in the tile: shared addresses are those of the round's
+// exchange tile, already offset to the thread's column pair.
+struct BlockPos {
+  uint32_t own;    // row i0 of the exchange tile
+  uint32_t prev;   // in-register rounds: the row just after the S source rows (row i0; row n for block 0)
+  uint32_t col;    // row 0
+  int i0, cnt, n;
+  bool full_block, publish;
+};
+
+// One round with a compile-time shift S smaller than every block.  Z (the payload) is Ih or Jh itself.
 template <int CB, int S, bool PAYJ>
-__device__ __forceinline__ void round_partial(float2 (&Ih)[CB], float2 (&Jh)[CB], float2 cI, float2 cJ, float *buf,
-                                              bool publish, bool full_block, int i0, int src_row0) {
-  float2(&Z)[CB] = PAYJ ? Jh : Ih;
-  if (publish) {
+__device__ __forceinline__ void round_partial(pk2 (&Ih)[CB], pk2 (&Jh)[CB], pk2 cI, pk2 cJ, const BlockPos &q) {
+  pk2(&Z)[CB] = PAYJ ? Jh : Ih;
+  if (q.publish) {
     // the last S rows of the block are what the next block's first S rows receive
-    float2 *own = reinterpret_cast<float2 *>(buf + i0 * kBkTileCols);
-    if (full_block) {
-#pragma unroll
-      for (int t = 0; t < S; ++t) own[(CB - S + t) * (kBkTileCols / 2)] = Z[CB - S + t];
+    if (q.full_block) {
+      static_for<S>([&](auto T) { sts64<(CB - S + CECA_IDX(T)) * kBkRowBytes>(q.own, Z[CB - S + CECA_IDX(T)]); });
     } else if constexpr (CB - 1 - S >= 0) {
-#pragma unroll
-      for (int t = 0; t < S; ++t) own[(CB - 1 - S + t) * (kBkTileCols / 2)] = Z[CB - 1 - S + t];
+      static_for<S>([&](auto T) { sts64<(CB - 1 - S + CECA_IDX(T)) * kBkRowBytes>(q.own, Z[CB - 1 - S + CECA_IDX(T)]); });
     }
     __syncthreads();
   }
-  float2 R[S];
-  const float2 *src = reinterpret_cast<const float2 *>(buf + src_row0 * kBkTileCols);  // S rows, no wrap inside
-#pragma unroll
-  for (int t = 0; t < S; ++t) R[t] = src[t * (kBkTileCols / 2)];
 #pragma unroll
   for (int j = CB - 1; j >= S; --j) {  // descending: Z[j - S] is still the value from before this round
-    const float2 z = Z[j - S];
+    const pk2 z = Z[j - S];
     Ih[j] = axpy2(cI, z, Ih[j]);
     Jh[j] = axpy2(cJ, z, Jh[j]);
   }
+  // the first S rows receive from the S rows before the block (no wrap inside), eight loads in flight at a time
+  constexpr int kChunk = 8;
+  static_for<(S + kChunk - 1) / kChunk>([&](auto C) {
+    constexpr int T0 = CECA_IDX(C) * kChunk;
+    constexpr int TN = S - T0 < kChunk ? S - T0 : kChunk;
+    pk2 R[TN];
+    static_for<TN>([&](auto T) { R[CECA_IDX(T)] = lds64<(T0 + CECA_IDX(T) - S) * kBkRowBytes>(q.prev); });
+    static_for<TN>([&](auto T) {
+      Ih[T0 + CECA_IDX(T)] = axpy2(cI, R[CECA_IDX(T)], Ih[T0 + CECA_IDX(T)]);
+      Jh[T0 + CECA_IDX(T)] = axpy2(cJ, R[CECA_IDX(T)], Jh[T0 + CECA_IDX(T)]);
+    });
+  });
+}
+
+// One round in which every row receives through shared memory (s at least as large as a block).
+template <int CB, bool PAYJ>
+__device__ __forceinline__ void round_full(pk2 (&Ih)[CB], pk2 (&Jh)[CB], pk2 cI, pk2 cJ, const BlockPos &q, int s) {
+  pk2(&Z)[CB] = PAYJ ? Jh : Ih;
+  if (q.publish) {
+    static_for<CB - 1>([&](auto J) { sts64<CECA_IDX(J) * kBkRowBytes>(q.own, Z[CECA_IDX(J)]); });
+    if (q.full_block) sts64<(CB - 1) * kBkRowBytes>(q.own, Z[CB - 1]);
+    __syncthreads();
+  }
+  const int first = q.i0 - s;  // source row of offset 0, before the wrap-around
+  if (first >= 0 || first + q.cnt <= 0) {  // the whole block on one side of the wrap-around
+    const uint32_t src = q.col + (uint32_t)((first >= 0 ? first : first + q.n) * kBkRowBytes);
+    constexpr int kChunk = 8;
+    static_for<(CB + kChunk - 1) / kChunk>([&](auto C) {
+      constexpr int J0 = CECA_IDX(C) * kChunk;
+      constexpr int JN = CB - J0 < kChunk ? CB - J0 : kChunk;
+      pk2 R[JN];
+      static_for<JN>([&](auto J) {
+        constexpr int row = J0 + CECA_IDX(J);
+        if constexpr (row < CB - 1) R[CECA_IDX(J)] = lds64<row * kBkRowBytes>(src);
+        else R[CECA_IDX(J)] = q.full_block ? lds64<row * kBkRowBytes>(src) : 0ull;
+      });
+      static_for<JN>([&](auto J) {
+        Ih[J0 + CECA_IDX(J)] = axpy2(cI, R[CECA_IDX(J)], Ih[J0 + CECA_IDX(J)]);
+        Jh[J0 + CECA_IDX(J)] = axpy2(cJ, R[CECA_IDX(J)], Jh[J0 + CECA_IDX(J)]);
+      });
+    });
+  } else {
 #pragma unroll
-  for (int t = 0; t < S; ++t) {
-    Ih[t] = axpy2(cI, R[t], Ih[t]);
-    Jh[t] = axpy2(cJ, R[t], Jh[t]);
+    for (int j = 0; j < CB; ++j) {
+      int row = first + j;
+      if (row < 0) row += q.n;
+      const pk2 r = (j < q.cnt) ? lds64<0>(q.col + (uint32_t)(row * kBkRowBytes)) : 0ull;
+      Ih[j] = axpy2(cI, r, Ih[j]);
+      Jh[j] = axpy2(cJ, r, Jh[j]);
+    }
   }
 }
 
-template <int CB, bool PAYJ>
-__device__ __forceinline__ void dispatch_partial(int s, float2 (&Ih)[CB], float2 (&Jh)[CB], float2 cI, float2 cJ,
-                                                 float *buf, bool publish, bool full_block, int i0, int src_row0) {
-#define CECA_BK_CASE(S)                                                                             \
-  case S:                                                                                           \
-    if constexpr (S < CB) round_partial<CB, S, PAYJ>(Ih, Jh, cI, cJ, buf, publish, full_block, i0, src_row0); \
+// `sel` (formed on the host): 0 / 1 = every row through shared memory, payload I / J;
+// 2 S + (0 / 1) = the in-register form with shift S, payload I / J.
+template <int CB>
+__device__ __forceinline__ void dispatch_round(int sel, int s, pk2 (&Ih)[CB], pk2 (&Jh)[CB], pk2 cI, pk2 cJ,
+                                               const BlockPos &q) {
+#define CECA_BK_CASE(S)                                                              \
+  case 2 * S:                                                                        \
+    if constexpr (S < CB) round_partial<CB, S, false>(Ih, Jh, cI, cJ, q);            \
+    break;                                                                           \
+  case 2 * S + 1:                                                                    \
+    if constexpr (S < CB) round_partial<CB, S, true>(Ih, Jh, cI, cJ, q);             \
     break;
-  switch (s) {
+  switch (sel) {
+    case 0: round_full<CB, false>(Ih, Jh, cI, cJ, q, s); break;
+    case 1: round_full<CB, true>(Ih, Jh, cI, cJ, q, s); break;
     CECA_BK_CASE(1) CECA_BK_CASE(2) CECA_BK_CASE(3) CECA_BK_CASE(4) CECA_BK_CASE(5) CECA_BK_CASE(6) CECA_BK_CASE(7)
     CECA_BK_CASE(8) CECA_BK_CASE(9) CECA_BK_CASE(10) CECA_BK_CASE(11) CECA_BK_CASE(12) CECA_BK_CASE(13)
-    CECA_BK_CASE(14) CECA_BK_CASE(15)
+    CECA_BK_CASE(14) CECA_BK_CASE(15) CECA_BK_CASE(16) CECA_BK_CASE(17) CECA_BK_CASE(18) CECA_BK_CASE(19)
+    CECA_BK_CASE(20) CECA_BK_CASE(21) CECA_BK_CASE(22) CECA_BK_CASE(23) CECA_BK_CASE(24)
     default: break;
   }
 #undef CECA_BK_CASE
 }
 
-// One round in which every row receives through shared memory (s at least as large as a block).
-template <int CB, bool PAYJ>
-__device__ __forceinline__ void round_full(float2 (&Ih)[CB], float2 (&Jh)[CB], float2 cI, float2 cJ, float *buf,
-                                           bool publish, bool full_block, int i0, int s, int n) {
-  float2(&Z)[CB] = PAYJ ? Jh : Ih;
-  if (publish) {
-    float2 *own = reinterpret_cast<float2 *>(buf + i0 * kBkTileCols);
-#pragma unroll
-    for (int j = 0; j < CB - 1; ++j) own[j * (kBkTileCols / 2)] = Z[j];
-    if (full_block) own[(CB - 1) * (kBkTileCols / 2)] = Z[CB - 1];
-    __syncthreads();
-  }
-  const int cnt = full_block ? CB : CB - 1;
-  const int first = i0 - s;  // source row of offset 0, before the wrap-around
-  float2 R[CB];
-  if (first >= 0 || first + cnt <= 0) {  // the whole block on one side of the wrap-around
-    const float2 *src = reinterpret_cast<const float2 *>(buf + (first >= 0 ? first : first + n) * kBkTileCols);
-#pragma unroll
-    for (int j = 0; j < CB - 1; ++j) R[j] = src[j * (kBkTileCols / 2)];
-    R[CB - 1] = full_block ? src[(CB - 1) * (kBkTileCols / 2)] : make_float2(0.f, 0.f);
-  } else {
-#pragma unroll
-    for (int j = 0; j < CB; ++j) {
-      int row = first + j;
-      if (row < 0) row += n;
-      R[j] = (j < cnt) ? *reinterpret_cast<const float2 *>(buf + row * kBkTileCols) : make_float2(0.f, 0.f);
-    }
-  }
-#pragma unroll
-  for (int j = 0; j < CB; ++j) {
-    Ih[j] = axpy2(cI, R[j], Ih[j]);
-    Jh[j] = axpy2(cJ, R[j], Jh[j]);
-  }
-}
-
-// MINB = CTAs per SM the register allocation must allow.
-template <int CB, int P, int MINB>
-__global__ void __launch_bounds__(32 * P, MINB)
+// The number of warps (blocks of agents) per CTA is a launch parameter; MAXT only bounds it and
+// thereby sets the register budget (65536 / MAXT registers per thread).
+template <int CB, int MAXT>
+__global__ void __launch_bounds__(MAXT, 1)
 consensus_block_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_y,
                        const __grid_constant__ BlockArgs p) {
   extern __shared__ __align__(128) unsigned char smem_raw[];
   __shared__ __align__(8) uint64_t bar;
   const int n = p.n;
   const int lane = threadIdx.x & 31, part = threadIdx.x >> 5;
-  const int tile_floats = n * kBkTileCols;
-  float *land_x = reinterpret_cast<float *>(smem_raw);   // [n][64] landed X tile
-  float *xch_a = land_x + tile_floats;                   // [n][64] exchange tile of the odd rounds
-  float *xch_b = xch_a + tile_floats;                    // [n][64] exchange tile of the even rounds
-  float *land_y = xch_b + tile_floats;                   // [n][64] landed Y tile (only when Y is read)
+  const uint32_t tile_bytes = (uint32_t)n * kBkRowBytes;
+  // [n][64] tiles: landed X, exchange tile of the odd rounds, of the even rounds (the same tile when
+  // there is only one), landed Y (when Y is read)
+  const uint32_t sm_land_x = smem_u32(smem_raw);
+  const uint32_t sm_xch_a = sm_land_x + tile_bytes, sm_xch_b = p.single_xch ? sm_xch_a : sm_xch_a + tile_bytes;
+  const uint32_t y_tile = p.single_xch ? 2u : 3u;
+  const uint32_t sm_land_y = sm_land_x + y_tile * tile_bytes;
 
-  const bool full_block = part < p.nfull;
-  const int cnt = full_block ? CB : CB - 1;
-  const int i0 = full_block ? part * CB : p.nfull * CB + (part - p.nfull) * (CB - 1);
-  const int colpair = 2 * lane;
+  BlockPos q;
+  q.n = n;
+  q.full_block = part < p.nfull;
+  q.cnt = q.full_block ? CB : CB - 1;
+  q.i0 = q.full_block ? part * CB : p.nfull * CB + (part - p.nfull) * (CB - 1);
+  const uint32_t col_off = 2u * lane * (uint32_t)sizeof(float);
+  const uint32_t own_off = (uint32_t)q.i0 * kBkRowBytes + col_off;
+  const uint32_t prev_off = (uint32_t)(part == 0 ? n : q.i0) * kBkRowBytes + col_off;
 
   if (threadIdx.x == 0) {
     mbar_init(&bar, 1);
@@ -189,10 +267,14 @@ consensus_block_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
 
   auto issue_load = [&](int32_t tile) {
     mbar_expect_tx(&bar, p.tx_bytes);
-    tma_load_2d(land_x, &map_x, tile * kBkTileCols, 0, &bar);
-    if (p.has_y_in) tma_load_2d(land_y, &map_y, tile * kBkTileCols, 0, &bar);
+    tma_load_2d(smem_raw, &map_x, tile * kBkTileCols, 0, &bar);
+    if (p.has_y_in) tma_load_2d(smem_raw + (size_t)y_tile * tile_bytes, &map_y, tile * kBkTileCols, 0, &bar);
   };
   if (threadIdx.x == 0 && (int32_t)blockIdx.x < p.tiles) issue_load((int32_t)blockIdx.x);
+
+  const bool prefetch_in_loop = p.rounds > 2;
+  float *const dst_x = p.Xo + (int64_t)q.i0 * p.ld + 2 * lane;
+  float *const dst_y = p.Yo + (int64_t)q.i0 * p.ld + 2 * lane;
 
   uint32_t phase = 0;
   for (int32_t tile = blockIdx.x; tile < p.tiles; tile += gridDim.x) {
@@ -207,79 +289,72 @@ consensus_block_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
     }
     phase ^= 1u;
 
-    float2 Ih[CB], Jh[CB];
+    pk2 Ih[CB], Jh[CB];
     {
-      const float2 *own = reinterpret_cast<const float2 *>(land_x + i0 * kBkTileCols + colpair);
-#pragma unroll
-      for (int j = 0; j < CB - 1; ++j) Ih[j] = own[j * (kBkTileCols / 2)];
-      Ih[CB - 1] = full_block ? own[(CB - 1) * (kBkTileCols / 2)] : make_float2(0.f, 0.f);
+      const uint32_t own = sm_land_x + own_off;
+      static_for<CB - 1>([&](auto J) { Ih[CECA_IDX(J)] = lds64<CECA_IDX(J) * kBkRowBytes>(own); });
+      Ih[CB - 1] = q.full_block ? lds64<(CB - 1) * kBkRowBytes>(own) : 0ull;
       if (p.has_y_in) {
-        const float2 *owny = reinterpret_cast<const float2 *>(land_y + i0 * kBkTileCols + colpair);
-#pragma unroll
-        for (int j = 0; j < CB - 1; ++j) Jh[j] = owny[j * (kBkTileCols / 2)];
-        Jh[CB - 1] = full_block ? owny[(CB - 1) * (kBkTileCols / 2)] : make_float2(0.f, 0.f);
+        const uint32_t owny = sm_land_y + own_off;
+        static_for<CB - 1>([&](auto J) { Jh[CECA_IDX(J)] = lds64<CECA_IDX(J) * kBkRowBytes>(owny); });
+        Jh[CB - 1] = q.full_block ? lds64<(CB - 1) * kBkRowBytes>(owny) : 0ull;
       } else {
 #pragma unroll
-        for (int j = 0; j < CB; ++j) Jh[j] = make_float2(0.f, 0.f);
+        for (int j = 0; j < CB; ++j) Jh[j] = 0ull;
       }
     }
     const int32_t next_tile = tile + (int32_t)gridDim.x;
-    const bool prefetch_in_loop = p.rounds > 2;
 
     for (int rnd = 0; rnd < p.rounds; ++rnd) {
       const BlockRound &rd = p.rd[rnd];
-      if (rd.renorm) {
-        const float sI = rd.preI, sJ = rd.preJ;
+      const int mode = rd.mode;
+      if (mode & (kBkRenorm | kBkClearJ)) {
+        if (mode & kBkRenorm) {
+          const pk2 sI = pk_make(rd.preI, rd.preI), sJ = pk_make(rd.preJ, rd.preJ);
 #pragma unroll
-        for (int j = 0; j < CB; ++j) { Ih[j].x *= sI; Ih[j].y *= sI; Jh[j].x *= sJ; Jh[j].y *= sJ; }
-      }
-      if (rd.jclear) {
+          for (int j = 0; j < CB; ++j) { Ih[j] = mul2(sI, Ih[j]); Jh[j] = mul2(sJ, Jh[j]); }
+        }
+        if (mode & kBkClearJ) {
 #pragma unroll
-        for (int j = 0; j < CB; ++j) Jh[j] = make_float2(0.f, 0.f);
+          for (int j = 0; j < CB; ++j) Jh[j] = 0ull;
+        }
       }
       if (rnd == 2 && threadIdx.x == 0 && next_tile < p.tiles) {
         // every thread has passed the barrier of round 1, so all reads of the landed tile (own rows and
         // the first round's neighbours) are done: the next tile may land while this one is finished
         issue_load(next_tile);
       }
-      const bool publish = rnd > 0;
-      float *buf = (rnd == 0 ? (rd.payload ? land_y : land_x) : ((rnd & 1) ? xch_a : xch_b)) + colpair;
-      const int s = rd.hop;
-      const float2 cI = make_float2(rd.cI, rd.cI), cJ = make_float2(rd.cJ, rd.cJ);
-      if (rd.partial) {
-        const int src_row0 = (part == 0 ? n : i0) - s;
-        if (rd.payload) dispatch_partial<CB, true>(s, Ih, Jh, cI, cJ, buf, publish, full_block, i0, src_row0);
-        else            dispatch_partial<CB, false>(s, Ih, Jh, cI, cJ, buf, publish, full_block, i0, src_row0);
-      } else {
-        if (rd.payload) round_full<CB, true>(Ih, Jh, cI, cJ, buf, publish, full_block, i0, s, n);
-        else            round_full<CB, false>(Ih, Jh, cI, cJ, buf, publish, full_block, i0, s, n);
-      }
+      // The first round finds every row's payload in the landed tile and publishes nothing.
+      q.publish = rnd > 0;
+      const uint32_t buf = rnd == 0 ? ((mode & kBkPayloadJ) ? sm_land_y : sm_land_x) : ((rnd & 1) ? sm_xch_a : sm_xch_b);
+      q.own = buf + own_off;
+      q.prev = buf + prev_off;
+      q.col = buf + col_off;
+      dispatch_round<CB>(rd.sel, rd.hop, Ih, Jh, pk_make(rd.cI, rd.cI), pk_make(rd.cJ, rd.cJ), q);
+      // with a single exchange tile the next round's publish must wait for this round's reads
+      if (p.single_xch && rnd >= 1 && rnd + 1 < p.rounds) __syncthreads();
     }
 
-    const int32_t col = tile * kBkTileCols + colpair;
-    if (col < p.d) {
-      const float oI = p.outI, oJ = p.outJ;
-      const bool pair_ok = col + 1 < p.d;   // d odd: the last column has no partner
-      float *dst = p.Xo + (int64_t)i0 * p.ld + col;
-      float *dsty = p.Yo + (int64_t)i0 * p.ld + col;
+    const int32_t col = tile * kBkTileCols + 2 * lane;
+    if (col + 1 < p.d) {
+      const pk2 oI = pk_make(p.outI, p.outI), oJ = pk_make(p.outJ, p.outJ);
+      float *dst = dst_x + col - 2 * lane;
 #pragma unroll
-      for (int j = 0; j < CB; ++j) {
-        if (j < CB - 1 || full_block) {
-          const float2 v = make_float2(oI * Ih[j].x, oI * Ih[j].y);
-          if (pair_ok) __stcs(reinterpret_cast<float2 *>(dst + j * p.ld), v);
-          else __stcs(dst + j * p.ld, v.x);
-        }
-      }
+      for (int j = 0; j < CB - 1; ++j) __stcs(reinterpret_cast<pk2 *>(dst + j * p.ld), mul2(oI, Ih[j]));
+      if (q.full_block) __stcs(reinterpret_cast<pk2 *>(dst + (CB - 1) * p.ld), mul2(oI, Ih[CB - 1]));
       if (p.has_y_out) {
+        float *dsty = dst_y + col - 2 * lane;
 #pragma unroll
-        for (int j = 0; j < CB; ++j) {
-          if (j < CB - 1 || full_block) {
-            const float2 v = make_float2(oJ * Jh[j].x, oJ * Jh[j].y);
-            if (pair_ok) __stcs(reinterpret_cast<float2 *>(dsty + j * p.ld), v);
-            else __stcs(dsty + j * p.ld, v.x);
-          }
-        }
+        for (int j = 0; j < CB - 1; ++j) __stcs(reinterpret_cast<pk2 *>(dsty + j * p.ld), mul2(oJ, Jh[j]));
+        if (q.full_block) __stcs(reinterpret_cast<pk2 *>(dsty + (CB - 1) * p.ld), mul2(oJ, Jh[CB - 1]));
       }
+    } else if (col < p.d) {   // d odd: the last column has no partner
+#pragma unroll
+      for (int j = 0; j < CB; ++j)
+        if (j < q.cnt) {
+          __stcs(p.Xo + (int64_t)(q.i0 + j) * p.ld + col, p.outI * pk_lo(Ih[j]));
+          if (p.has_y_out) __stcs(p.Yo + (int64_t)(q.i0 + j) * p.ld + col, p.outJ * pk_lo(Jh[j]));
+        }
     }
     if (!prefetch_in_loop && next_tile < p.tiles) {
       // fewer than three rounds: the landed tile was in use until the end
@@ -294,38 +369,90 @@ consensus_block_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
 constexpr int kBkMaxRows = 256;
 constexpr size_t kBkSmemLimit = 227 * 1024 - 1024;   // opt-in maximum per CTA minus the static part
 
-// y_in: the first round reads Y, which takes a fourth shared-memory tile.
+// y_in: the first round reads Y, which takes one more shared-memory tile (at least two are needed without it).
 bool consensus_block_supports(int32_t n, ceca_variant_t variant, int32_t rounds, bool y_in) {
   return variant == CECA_2P && n >= 2 && n <= kBkMaxRows && rounds >= 1 && rounds <= kBkMaxRounds &&
-         (size_t)(y_in ? 4 : 3) * n * kBkTileCols * sizeof(float) <= kBkSmemLimit;
+         (size_t)(y_in ? 3 : 2) * n * kBkTileCols * sizeof(float) <= kBkSmemLimit;
 }
 
-template <int CB, int P, int MINB>
-static cudaError_t launch_block(const CUtensorMap &mx, const CUtensorMap &my, BlockArgs &a, cudaStream_t stream) {
-  const int n = a.n;
-  a.nfull = n - P * (CB - 1);
-  const int cmin = a.nfull == P ? CB : CB - 1;
-  for (int t = 0; t < a.rounds; ++t) a.rd[t].partial = (a.rd[t].hop < cmin) ? 1 : 0;
-  const size_t tile_bytes = (size_t)n * kBkTileCols * sizeof(float);
-  const size_t smem = (a.has_y_in ? 4 : 3) * tile_bytes;
-  constexpr size_t kMaxSmemWanted = (size_t)4 * CB * P * kBkTileCols * sizeof(float);
-  constexpr size_t kMaxSmem = kMaxSmemWanted < kBkSmemLimit ? kMaxSmemWanted : kBkSmemLimit;
-  if (smem > kMaxSmem) return cudaErrorInvalidConfiguration;
+constexpr int kBkMaxWarps = 12;   // 12 blocks of 22 agents cover n = 256
+
+// Register budgets by block size (the state takes 4 * CB registers): a roomy one, and a lean one that
+// still compiles without spilling to speak of.  65536 / kMaxThreads registers per thread.
+template <int CB> struct BlockRegs {
+  static constexpr int kRoomy = CB >= 15 ? 384 : CB >= 11 ? 640 : CB >= 7 ? 768 : 1024;
+  static constexpr int kLean = CB >= 15 ? 512 : CB >= 11 ? 768 : 1024;
+};
+
+template <int CB, int MAXT>
+static cudaError_t launch_block_regs(const CUtensorMap &mx, const CUtensorMap &my, const BlockArgs &a, int warps,
+                                     size_t smem, int *per_sm_out, bool launch, cudaStream_t stream) {
   static std::atomic<uint64_t> attr_done{0};
-  cudaError_t e =
-      set_max_shared_once(reinterpret_cast<const void *>(consensus_block_kernel<CB, P, MINB>), kMaxSmem, &attr_done);
+  cudaError_t e = set_max_shared_once(reinterpret_cast<const void *>(consensus_block_kernel<CB, MAXT>), kBkSmemLimit,
+                                      &attr_done);
   if (e != cudaSuccess) return e;
+  int per_sm = 0;
+  e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, consensus_block_kernel<CB, MAXT>, 32 * warps, smem);
+  if (e != cudaSuccess) return e;
+  *per_sm_out = per_sm;
+  if (!launch) return cudaSuccess;
+  if (per_sm < 1) return cudaErrorInvalidConfiguration;
   const int sms = sm_count();
   if (sms <= 0) return cudaErrorUnknown;
   // persistent CTAs: as many as fit on the device at once, not more than there are tiles
-  int per_sm = 0;
-  e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, consensus_block_kernel<CB, P, MINB>, 32 * P, smem);
-  if (e != cudaSuccess) return e;
-  if (per_sm < 1) return cudaErrorInvalidConfiguration;
   const int64_t resident = (int64_t)sms * per_sm;
   const int grid = (int)(a.tiles < resident ? a.tiles : resident);
-  consensus_block_kernel<CB, P, MINB><<<grid, 32 * P, smem, stream>>>(mx, my, a);
+  consensus_block_kernel<CB, MAXT><<<grid, 32 * warps, smem, stream>>>(mx, my, a);
   return cudaGetLastError();
+}
+
+template <int CB>
+static cudaError_t launch_block(const CUtensorMap &mx, const CUtensorMap &my, BlockArgs &a, int warps,
+                                cudaStream_t stream) {
+  const int n = a.n;
+  a.nfull = n - warps * (CB - 1);
+  const int cmin = a.nfull == warps ? CB : CB - 1;
+  for (int t = 0; t < a.rounds; ++t) {
+    BlockRound &r = a.rd[t];
+    const int pay = (r.mode & kBkPayloadJ) ? 1 : 0;
+    r.sel = r.hop < cmin ? 2 * r.hop + pay : pay;   // in-register form while the shift is smaller than every block
+  }
+  const size_t tile_bytes = (size_t)n * kBkTileCols * sizeof(float);
+  if (32 * warps > BlockRegs<CB>::kRoomy) return cudaErrorInvalidConfiguration;
+  // Four candidates: two or one exchange tile, roomy or lean register budget.  The default is two tiles
+  // and the roomy budget; an alternative is taken only when it lets more CTAs share an SM.
+  constexpr int kRoomy = BlockRegs<CB>::kRoomy, kLean = BlockRegs<CB>::kLean;
+  int best = 0, best_single = 0, best_lean = 0;
+  for (int single = 0; single < 2; ++single) {
+    const size_t smem = ((a.has_y_in ? 2 : 1) + (single ? 1 : 2)) * tile_bytes;
+    if (smem > kBkSmemLimit) continue;
+    int roomy = 0, lean = 0;
+    cudaError_t e = launch_block_regs<CB, kRoomy>(mx, my, a, warps, smem, &roomy, false, stream);
+    if (e != cudaSuccess) return e;
+    if (kLean != kRoomy) {
+      e = launch_block_regs<CB, kLean>(mx, my, a, warps, smem, &lean, false, stream);
+      if (e != cudaSuccess) return e;
+    }
+    if (roomy > best) { best = roomy; best_single = single; best_lean = 0; }
+    if (lean > best) { best = lean; best_single = single; best_lean = 1; }
+  }
+  if (best < 1) return cudaErrorInvalidConfiguration;
+  a.single_xch = best_single;
+  const size_t smem = ((a.has_y_in ? 2 : 1) + (best_single ? 1 : 2)) * tile_bytes;
+  int per_sm = 0;
+  if (best_lean) return launch_block_regs<CB, kLean>(mx, my, a, warps, smem, &per_sm, true, stream);
+  return launch_block_regs<CB, kRoomy>(mx, my, a, warps, smem, &per_sm, true, stream);
+}
+
+// Blocks (= warps) per CTA for n agents.  As few, i.e. as large, as the register file allows (25
+// agents take 100 state registers), because a round whose shift reaches the block size exchanges
+// every row through shared memory and there are about log2(blocks) such rounds; and 1, 2 or a
+// multiple of 4, so that the warps of a CTA, which move in lockstep from barrier to barrier, load
+// the four schedulers of an SM evenly (5, 6, 7 or 9 warps measured 15-40 % slower than 4 or 8).
+// `warps_override` > 0 forces a value (used to measure the alternatives).
+static int block_warps(int n, int warps_override) {
+  if (warps_override > 0) return warps_override;
+  return n <= 25 ? 1 : n <= 50 ? 2 : n <= 100 ? 4 : n <= 200 ? 8 : 12;
 }
 
 // Arguments are assumed validated by the caller (shapes, aliasing, 16-byte alignment of X / Y and
@@ -333,7 +460,7 @@ static cudaError_t launch_block(const CUtensorMap &mx, const CUtensorMap &my, Bl
 // The caller has checked consensus_block_supports.
 ceca_status_t consensus_block(const float *X, const float *Y, float *Xo, float *Yo, int32_t n, int64_t d,
                               int64_t ld, int64_t k0, int32_t rounds, int32_t *status, int32_t wait_polls,
-                              uint32_t tx_extra, cudaStream_t stream) {
+                              uint32_t tx_extra, int warps_override, cudaStream_t stream) {
   BlockArgs a;
   std::memset(&a, 0, sizeof(a));
   a.Xo = Xo; a.Yo = Yo; a.ld = ld; a.d = (int32_t)d; a.n = n; a.rounds = rounds;
@@ -351,15 +478,15 @@ ceca_status_t consensus_block(const float *X, const float *Y, float *Xo, float *
     if (t == 0) first_needs_y = plan.reads_y;
     BlockRound &r = a.rd[t];
     if (t > 0 && t % kBkRenormEvery == 0) {  // fold the scales back so that the scaled values stay in range
-      r.renorm = 1; r.preI = (float)alpha; r.preJ = (float)beta;
+      r.mode |= kBkRenorm; r.preI = (float)alpha; r.preJ = (float)beta;
       alpha = 1.0; beta = 1.0;
     }
     const double wa = plan.rd.a, wb = plan.rd.b;
     const double zeta = plan.rd.payload ? beta : alpha;
-    r.payload = (uint8_t)plan.rd.payload;
-    r.hop = (int16_t)plan.walk.hop;
+    if (plan.rd.payload) r.mode |= kBkPayloadJ;
+    r.hop = plan.walk.hop;
     r.cI = (float)((1.0 - wa) * zeta / (wa * alpha));
-    if (plan.rd.b_num == 0) { r.jclear = 1; r.cJ = 1.f; }   // J+ = the received value: Jh = 0 + 1 * zh_src, beta+ = zeta
+    if (plan.rd.b_num == 0) { r.mode |= kBkClearJ; r.cJ = 1.f; }   // J+ = the received value: Jh = 0 + 1 * zh_src, beta+ = zeta
     else r.cJ = (float)((1.0 - wb) * zeta / (wb * beta));
     alpha = wa * alpha;
     beta = plan.rd.b_num == 0 ? zeta : wb * beta;
@@ -373,37 +500,18 @@ ceca_status_t consensus_block(const float *X, const float *Y, float *Xo, float *
   if (!tensor_map_2d(&mx, X, n, d, ld, kBkTileCols, n)) return CECA_ERR_CUDA;
   if (!tensor_map_2d(&my, a.has_y_in ? Y : X, n, d, ld, kBkTileCols, n)) return CECA_ERR_CUDA;
 
-  cudaError_t e = cudaErrorInvalidValue;
-  if (n <= 8 * kBkMaxCb) {
-    switch ((n + 7) / 8) {   // 8 warps, blocks of ceil(n / 8) agents
-      case 1: e = launch_block<1, 8, 4>(mx, my, a, stream); break;
-      case 2: e = launch_block<2, 8, 4>(mx, my, a, stream); break;
-      case 3: e = launch_block<3, 8, 4>(mx, my, a, stream); break;
-      case 4: e = launch_block<4, 8, 4>(mx, my, a, stream); break;
-      case 5: e = launch_block<5, 8, 4>(mx, my, a, stream); break;
-      case 6: e = launch_block<6, 8, 4>(mx, my, a, stream); break;
-      case 7: e = launch_block<7, 8, 3>(mx, my, a, stream); break;
-      case 8: e = launch_block<8, 8, 3>(mx, my, a, stream); break;
-      case 9: e = launch_block<9, 8, 3>(mx, my, a, stream); break;
-      case 10: e = launch_block<10, 8, 3>(mx, my, a, stream); break;
-      case 11: e = launch_block<11, 8, 2>(mx, my, a, stream); break;
-      case 12: e = launch_block<12, 8, 2>(mx, my, a, stream); break;
-      case 13: e = launch_block<13, 8, 2>(mx, my, a, stream); break;
-      case 14: e = launch_block<14, 8, 2>(mx, my, a, stream); break;
-      case 15: e = launch_block<15, 8, 2>(mx, my, a, stream); break;
-      case 16: e = launch_block<16, 8, 2>(mx, my, a, stream); break;
-    }
-  } else {
-    switch ((n + 15) / 16) {  // 16 warps, n = 129 .. 256
-      case 9: e = launch_block<9, 16, 1>(mx, my, a, stream); break;
-      case 10: e = launch_block<10, 16, 1>(mx, my, a, stream); break;
-      case 11: e = launch_block<11, 16, 1>(mx, my, a, stream); break;
-      case 12: e = launch_block<12, 16, 1>(mx, my, a, stream); break;
-      case 13: e = launch_block<13, 16, 1>(mx, my, a, stream); break;
-      case 14: e = launch_block<14, 16, 1>(mx, my, a, stream); break;
-      case 15: e = launch_block<15, 16, 1>(mx, my, a, stream); break;
-      case 16: e = launch_block<16, 16, 1>(mx, my, a, stream); break;
-    }
+  const int warps = block_warps(n, warps_override);
+  if (warps < 1 || warps > kBkMaxWarps) return CECA_ERR_UNSUPPORTED;
+  cudaError_t e = cudaErrorInvalidConfiguration;
+  switch ((n + warps - 1) / warps) {   // agents per block
+#define CECA_BK_LAUNCH(CB) case CB: e = launch_block<CB>(mx, my, a, warps, stream); break;
+    CECA_BK_LAUNCH(1) CECA_BK_LAUNCH(2) CECA_BK_LAUNCH(3) CECA_BK_LAUNCH(4) CECA_BK_LAUNCH(5) CECA_BK_LAUNCH(6)
+    CECA_BK_LAUNCH(7) CECA_BK_LAUNCH(8) CECA_BK_LAUNCH(9) CECA_BK_LAUNCH(10) CECA_BK_LAUNCH(11) CECA_BK_LAUNCH(12)
+    CECA_BK_LAUNCH(13) CECA_BK_LAUNCH(14) CECA_BK_LAUNCH(15) CECA_BK_LAUNCH(16) CECA_BK_LAUNCH(17) CECA_BK_LAUNCH(18)
+    CECA_BK_LAUNCH(19) CECA_BK_LAUNCH(20) CECA_BK_LAUNCH(21) CECA_BK_LAUNCH(22) CECA_BK_LAUNCH(23) CECA_BK_LAUNCH(24)
+    CECA_BK_LAUNCH(25)
+#undef CECA_BK_LAUNCH
+    default: break;
   }
   if (e == cudaErrorInvalidConfiguration) return CECA_ERR_UNSUPPORTED;
   return e == cudaSuccess ? CECA_OK : CECA_ERR_CUDA;

@@ -266,7 +266,7 @@ def _fused_kernels(n, variant=ceca.CECA_2P):
     kernels = [ceca.FUSED_SMEM]
     if n <= 128:
         kernels.append(ceca.FUSED_TMEM)
-    if n <= 226 and variant == ceca.CECA_2P:   # (up to 256 when the first round does not read Y)
+    if n <= 256 and variant == ceca.CECA_2P:
         kernels.append(ceca.FUSED_BLOCK)
     return kernels
 
@@ -290,11 +290,6 @@ def test_consensus_matches_oracle_and_reaches_the_mean(fused, n, d):
             X, Y = x.to(DEV), y0.to(DEV)
             Xo, Yo = torch.empty_like(X), torch.empty_like(Y)
             ws = _fused_ws()
-            if fused == ceca.FUSED_BLOCK and n > 226 and k0 % tau:
-                # a first round that reads Y needs a fourth shared-memory tile, which no longer fits
-                with pytest.raises(ceca.CecaError):
-                    ceca.ceca_consensus_rounds(X, Y, variant, k0, rounds, fused, X_out=Xo, Y_out=Yo, workspace=ws)
-                continue
             ceca.ceca_consensus_rounds(X, Y, variant, k0, rounds, fused, X_out=Xo, Y_out=Yo, workspace=ws)
             assert ceca.ceca_read_status(ws) == 0
             want_x, want_y = oracle.consensus(_np(x), _np(y0), variant, k0, rounds)
