@@ -39,6 +39,9 @@ WORKLOADS = {
     "resnet50_step": dict(kind="step", n=100, d=25_557_032, variant=2, gamma=0.1),
     # the same, but the caller declines the dead y+ of the last round of each cycle (one write less in 1 of 7 steps)
     "resnet50_step_dead_y": dict(kind="step", n=100, d=25_557_032, variant=2, gamma=0.1, drop_dead_y=True),
+    # narrower storage, fp32 arithmetic (not in the paper): G as bf16 (18 B per agent-parameter), or X, Y, G as bf16 (10 B)
+    "resnet50_step_g_bf16": dict(kind="step", n=100, d=25_557_032, variant=2, gamma=0.1, storage="g_bf16"),
+    "resnet50_step_bf16": dict(kind="step", n=100, d=25_557_032, variant=2, gamma=0.1, storage="bf16"),
     # smaller cases of the same kernels, for profiler captures and quick looks
     "resnet18_step": dict(kind="step", n=24, d=11_689_512, variant=1, gamma=0.1),
     "step_small": dict(kind="step", n=100, d=2_097_152, variant=2, gamma=0.1),
@@ -245,15 +248,34 @@ def bench_step(args, wl, device, dist):
     n, d, variant, gamma = wl["n"], wl["d"], wl["variant"], wl["gamma"]
     ld = synth.padded_ld(d)  # rows 128-byte aligned: a warp's 512-byte access then covers exactly four lines
     X, Y, G = synth.step_inputs(n, d, seed=0, x_std=0.01, g_std=0.01, device=device, ld=ld)
+    storage = wl.get("storage", "f32")
+    if storage != "f32":   # the same draws, stored narrow (row by row: no second full-size temporary)
+        def narrow(t):
+            out = torch.empty((n, ld), dtype=torch.bfloat16, device=device)[:, :d]
+            for i in range(n):
+                out[i].copy_(t[i])
+            return out
+        G = narrow(G)
+        if storage == "bf16":
+            X, Y = narrow(X), narrow(Y)
+        torch.cuda.empty_cache()
+    bytes_reads_y, bytes_round0 = {"f32": (20, 16), "g_bf16": (18, 14), "bf16": (10, 8)}[storage]
     stream = torch.cuda.current_stream()
     tau = ceca.ceca_schedule(n, variant, 0, peers=False)[0].tau
     x_only = bool(wl.get("x_only"))
     if x_only:
         Y = None
     drop = bool(wl.get("drop_dead_y"))
+
+    def step(k):
+        if storage == "f32":
+            ceca.ceca_gossip_sgd_step(X, Y, G, gamma, variant, k, drop_y=drop and k % tau == tau - 1)
+        else:
+            ceca.ceca_gossip_sgd_step_bf16(X, Y, G, gamma, variant, k)
+
     k = 0
     for _ in range(args.warmup):
-        ceca.ceca_gossip_sgd_step(X, Y, G, gamma, variant, k, drop_y=drop and k % tau == tau - 1)
+        step(k)
         k += 1
     events = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
     k_first = k
@@ -264,7 +286,7 @@ def bench_step(args, wl, device, dist):
     torch.cuda.synchronize()
     events[0].record(stream)
     for s in range(args.steps):
-        ceca.ceca_gossip_sgd_step(X, Y, G, gamma, variant, k, drop_y=drop and k % tau == tau - 1)
+        step(k)
         k += 1
         events[s + 1].record(stream)
     torch.cuda.synchronize()
@@ -283,10 +305,13 @@ def bench_step(args, wl, device, dist):
     if dominant:
         avg_ms = sum(dominant) / len(dominant)
         peak, which = measured_peak()
-        achieved = (12 * n * d if x_only else algorithmic_bytes_step(n, d, True)) / (avg_ms * 1e-3) / 1e9
+        achieved = (12 if x_only else bytes_reads_y) * n * d / (avg_ms * 1e-3) / 1e9
         roof = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                 "traffic": ncu_traffic(args.workload),
-                "kernel": "step_walk_kernel<float4, gradient, %s>" % ("X only" if x_only else "reads Y"), "peak_source": "of " + which,
+                "kernel": "step_walk_kernel<%s, gradient, %s>" % (
+                    {"f32": "float4", "g_bf16": "float4, G bf16", "bf16": "8 columns, X Y G bf16"}[storage],
+                    "X only" if x_only else "reads Y"), "peak_source": "of " + which,
+                "bytes_per_agent_param": 12 if x_only else bytes_reads_y,
                 "avg_launch_ms": avg_ms, "median_launch_ms": statistics.median(dominant), "best_launch_ms": min(dominant),
                 "launches_timed": len(dominant),
                 "frac_of_nominal_8TBs": achieved / 8000.0,
@@ -294,8 +319,8 @@ def bench_step(args, wl, device, dist):
                                 if any((k_first + s) % tau == r for s in range(args.steps)) else None for r in range(tau)]}
     del X, Y, G
     torch.cuda.empty_cache()
-    return total_ms, launches, roof, clocks, {"tau": tau, "in_place": True, "ld": ld,
-                                               "l2": "inputs (3 x n x d fp32) far larger than L2"}
+    return total_ms, launches, roof, clocks, {"tau": tau, "in_place": True, "ld": ld, "storage": storage,
+                                               "l2": "inputs (3 arrays of n x d) far larger than L2"}
 
 
 def bench_step_e2e(args, wl, device):
@@ -545,16 +570,47 @@ def bench_sweep(args, wl, device, dist):
                                                "l2": "n >= 8 rows of 16.8 MB per array exceed L2; smaller n partly L2-resident"}
 
 
+SECONDARY = ["consensus_fused", "consensus_rounds", "consensus_fused_130", "consensus_fused_1026", "logreg_grad",
+             "resnet18_step"]
+
+
+def run_secondary(device, steps=20, warmup=5):
+    """Short legs of the other configurations, attached to the default line as `secondary`: the fused and the
+    per-round consensus at n = 97, the fused consensus at the paper's n = 130 and n = 1026, the logistic gradient
+    at n = 63, m = 2000, d = 4096 and the 1-port step at ResNet-18 size.  Each leg is the same function a
+    --workload run of that name calls, with its own inputs, warm-up and CUDA events."""
+    import torch
+    out = []
+    for name in SECONDARY:
+        wl = WORKLOADS[name]
+        sub = argparse.Namespace(steps=steps, warmup=warmup, workload=name)
+        fn = {"step": bench_step, "consensus": bench_consensus, "logreg": bench_logreg}[wl["kind"]]
+        try:
+            total_ms, launches, roof, clocks, _ = fn(sub, wl, device, None)
+        except Exception as exc:   # a leg that fails must not take the headline down with it
+            out.append({"workload": name, "error": "%s: %s" % (type(exc).__name__, exc)})
+            continue
+        ms = total_ms / steps
+        out.append({"workload": name, "n_agents": wl["n"], "d": wl["d"], "variant": "2P" if wl["variant"] == 2 else "1P",
+                    "steps": steps, "warmup": warmup, "ms_per_step": ms, "updates_per_s": wl["n"] * wl["d"] / (ms * 1e-3),
+                    "gpu_launches": launches, "clocks": clocks,
+                    "roofline": {k: roof[k] for k in ("bound", "achieved", "peak", "unit", "frac", "traffic", "kernel", "peak_source",
+                                                      "avg_launch_ms") if k in roof}})
+        torch.cuda.empty_cache()
+    return out
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=70)
+    ap.add_argument("--steps", type=int, default=70)    # ten cycles of the CECA sequence at n = 100 (tau = 7)
     ap.add_argument("--warmup", type=int, default=7)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="resnet50_step", choices=sorted(WORKLOADS))
     ap.add_argument("--e2e-steps", type=int, default=7)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-secondary", action="store_true")
     args = ap.parse_args()
     wl = WORKLOADS[args.workload]
 
@@ -586,7 +642,7 @@ def main():
         value = world * extra.pop("units") / (total_ms * 1e-3)
 
     e2e = None
-    if wl["kind"] == "step" and not args.no_e2e and not wl.get("x_only") and not wl.get("drop_dead_y"):
+    if wl["kind"] == "step" and not args.no_e2e and not wl.get("x_only") and not wl.get("drop_dead_y") and not wl.get("storage"):
         need = world * 3 * units_per_step * 4          # every rank keeps X, Y, G of its block in host memory
         avail = host_memory_available()
         if avail is not None and need > 0.7 * avail:
@@ -601,13 +657,17 @@ def main():
             e2e["value"] = world * units_per_step / (ms * 1e-3)
 
     cpu = None
-    if rank == 0 and world == 1 and wl["kind"] == "step" and not args.no_cpu_baseline:
+    if rank == 0 and world == 1 and wl["kind"] == "step" and not args.no_cpu_baseline and not wl.get("storage"):
         cols = min(wl["d"], 262_144)
         v, sec, threads = oracle_step_throughput(wl["n"], wl["variant"], wl["gamma"], cols, 3 * extra["tau"])
         v1, _, _ = oracle_step_throughput(wl["n"], wl["variant"], wl["gamma"], cols // 4, extra["tau"], threads=1)
         cpu = {"value": v, "unit": UNIT, "cores": threads, "kind": "oracle",
                "sample": "%d-column slice (all %d rows), %d steps = 3 cycles of the CECA sequence, fp64" % (cols, wl["n"], 3 * extra["tau"]),
                "single_thread_value": v1, "host_cores": os.cpu_count(), "cpu_model": cpu_model()}
+
+    secondary = None
+    if rank == 0 and world == 1 and args.workload == "resnet50_step" and not args.no_secondary:
+        secondary = run_secondary(device)
 
     if rank == 0:
         config = {"workload": args.workload, "n_agents": wl["n"], "d": wl["d"], "variant": "2P" if wl["variant"] == 2 else "1P"}
@@ -616,6 +676,8 @@ def main():
                 "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
                 "dtype": "f32", "data": "synthetic", "config": config, "clocks": clocks, "gpu_launches": launches,
                 "e2e": e2e, "roofline": roof, "cpu_baseline": cpu}
+        if secondary is not None:
+            line["secondary"] = secondary
         print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()

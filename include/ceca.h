@@ -106,6 +106,28 @@ ceca_status_t ceca_gossip_sgd_step(const float *X, const float *Y, const float *
                                    ceca_variant_t variant, int64_t k, void *stream);
 
 /*
+ * The same iteration with narrower storage (not in the paper, which only says that the update is
+ * "additions and scaling"; the kernel is bound by the bytes it moves, so narrower storage is the
+ * one way left to make it faster).  Arithmetic is fp32 in both forms; bf16 values are widened on
+ * load and rounded to nearest even on store.
+ *   xy_bf16 = 0: G is bf16 (n x d, leading dimension ld elements), X, Y, X_out, Y_out are fp32:
+ *                18 bytes per agent-parameter instead of 20.  The result is the fp32 update of the
+ *                gradient values as stored, to the same tolerance as ceca_gossip_sgd_step.
+ *   xy_bf16 = 1: X, Y, G, X_out, Y_out are all bf16: 10 bytes per agent-parameter.  Every stored
+ *                model value carries one bf16 rounding (relative 2^-9), so increments smaller than
+ *                that are lost and the 1e-5 consensus accuracy of the fp32 form is out of reach:
+ *                a bandwidth/accuracy trade the caller has to want.
+ * Pointers are device pointers to fp32 or bf16 elements as stated; ld counts elements of either.
+ * G and Y_out are required (no X-only or dead-y form); Y may be NULL where the round ignores it.
+ * Full-width accesses need ld % 4 == 0 (xy_bf16 = 0) or ld % 8 == 0 (xy_bf16 = 1) and 16-byte
+ * aligned fp32 / 8- resp. 16-byte aligned bf16 rows; anything else runs the scalar form.
+ * Aliasing rules and error codes as for ceca_gossip_sgd_step.
+ */
+ceca_status_t ceca_gossip_sgd_step_bf16(const void *X, const void *Y, const void *G, void *X_out, void *Y_out,
+                                        int32_t n, int64_t d, int64_t ld, int32_t xy_bf16, float gamma,
+                                        ceca_variant_t variant, int64_t k, void *stream);
+
+/*
  * `rounds` consecutive CECA rounds k0, k0+1, ..., k0+rounds-1 on (I, J) = (X, Y)
  * (Sec. 3.1 "Main recursions", Algorithm 2; Sec. 3.2 for the 1-port pairing).
  * After tau rounds that start at a multiple of tau every row of X_out is the column mean of

@@ -17,7 +17,7 @@ WS_STEP_HOST = 4
 EXPORTS = ["ceca_schedule", "ceca_gossip_sgd_step", "ceca_consensus_rounds", "dsgd_logreg_grad",
            "ceca_workspace_bytes", "ceca_read_status", "ceca_gossip_sgd_step_host", "ceca_status_string",
            "dsgd_logreg_grad_static", "dsgd_logreg_grad_static_capacity", "dsgd_lsq_grad",
-           "ceca_fused_wait_selftest"]
+           "ceca_fused_wait_selftest", "ceca_gossip_sgd_step_bf16"]
 
 
 class Round(ctypes.Structure):
@@ -54,6 +54,8 @@ def library():
     lib.ceca_schedule.restype = ctypes.c_int
     lib.ceca_gossip_sgd_step.argtypes = [vp, vp, vp, vp, vp, i32, i64, i64, f32, i32, i64, vp]
     lib.ceca_gossip_sgd_step.restype = ctypes.c_int
+    lib.ceca_gossip_sgd_step_bf16.argtypes = [vp, vp, vp, vp, vp, i32, i64, i64, i32, f32, i32, i64, vp]
+    lib.ceca_gossip_sgd_step_bf16.restype = ctypes.c_int
     lib.ceca_consensus_rounds.argtypes = [vp, vp, vp, vp, i32, i64, i64, i32, i64, i32, i32, vp,
                                           ctypes.c_size_t, vp]
     lib.ceca_consensus_rounds.restype = ctypes.c_int
@@ -137,6 +139,34 @@ def ceca_gossip_sgd_step(X, Y, G, gamma, variant, k, X_out=None, Y_out=None, str
     st = library().ceca_gossip_sgd_step(_ptr(X), _ptr(Y), _ptr(G), _ptr(X_out), _ptr(Y_out), n, d, ld,
                                         float(gamma), variant, k, _stream(stream))
     _check(st, "ceca_gossip_sgd_step")
+    return X_out, Y_out
+
+
+def _matrix_of(t, name, dtype, n=None):
+    """(n, d, ld) of a 2-D device tensor of the given dtype whose rows are contiguous."""
+    if t.dtype != dtype or t.dim() != 2 or t.stride(1) != 1 or not t.is_cuda:
+        raise ValueError("%s must be a 2-D %s device tensor with unit column stride" % (name, dtype))
+    if n is not None and t.shape[0] != n:
+        raise ValueError("%s has the wrong number of rows" % name)
+    return t.shape[0], t.shape[1], t.stride(0) if t.shape[0] > 1 else max(t.stride(0), t.shape[1])
+
+
+def ceca_gossip_sgd_step_bf16(X, Y, G, gamma, variant, k, X_out=None, Y_out=None, stream=None):
+    """One DSGD-CECA iteration with G stored as bfloat16 and X, Y either float32 or bfloat16 (all the same).
+    Outputs default to in place.  Returns (X_out, Y_out)."""
+    import torch
+    xy = X.dtype
+    if xy not in (torch.float32, torch.bfloat16):
+        raise ValueError("X must be float32 or bfloat16")
+    n, d, ld = _matrix_of(X, "X", xy)
+    X_out = X if X_out is None else X_out
+    Y_out = Y if Y_out is None else Y_out
+    for t, name, dt in ((Y, "Y", xy), (G, "G", torch.bfloat16), (X_out, "X_out", xy), (Y_out, "Y_out", xy)):
+        if t is not None and _matrix_of(t, name, dt, n) != (n, d, ld):
+            raise ValueError("%s must have the shape and row stride (in elements) of X" % name)
+    st = library().ceca_gossip_sgd_step_bf16(_ptr(X), _ptr(Y), _ptr(G), _ptr(X_out), _ptr(Y_out), n, d, ld,
+                                             int(xy == torch.bfloat16), float(gamma), variant, k, _stream(stream))
+    _check(st, "ceca_gossip_sgd_step_bf16")
     return X_out, Y_out
 
 

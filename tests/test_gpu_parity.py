@@ -725,6 +725,87 @@ def test_full_size_step_on_column_windows(n, d, variant, iters):
             assert np.abs(_np(X[:, lo:hi]) - ref[w][0]).max() <= tol * (k + 1)
 
 
+# --------------------------------------------------------------------------------------------
+# bf16 storage (fp32 arithmetic): the gradient alone, or X, Y and the gradient
+# --------------------------------------------------------------------------------------------
+
+BF16_HALF_ULP = 2.0 ** -8    # round-to-nearest into 8 significant bits: at most 2^-8 relative
+
+
+def _wide(t):
+    """The exact fp64 values of a float32 / bfloat16 tensor."""
+    return t.detach().float().cpu().numpy().astype(np.float64)
+
+
+def _bf16_tol(want, scale, xy_bf16):
+    """fp32 arithmetic on the stored values (2e-6 * scale, as for the fp32 step), plus one rounding of the
+    result to bfloat16 when the models are stored narrow."""
+    return STEP_TOL * scale + (BF16_HALF_ULP * np.abs(want) if xy_bf16 else 0.0)
+
+
+@pytest.mark.parametrize("xy_bf16", [False, True])
+@pytest.mark.parametrize("n,d,ld,offset", [(1, 9, 9, 0), (5, 37, 37, 0), (6, 64, 64, 0), (24, 1000, 1000, 0), (24, 1000, 1008, 8),
+                                            (24, 1001, 1004, 4), (97, 4100, 4104, 0), (100, 70001, 70008, 0)])
+def test_step_with_bf16_storage_matches_oracle(xy_bf16, n, d, ld, offset):
+    gamma = 0.1
+    x, y, g = synth.step_inputs(n, d, seed=n + d, x_std=1.0, g_std=1.0, same_xy=False)
+    xy_t = torch.bfloat16 if xy_bf16 else torch.float32
+
+    def put(src, dtype):
+        buf = torch.full((n * ld + offset + 16,), float("nan"), dtype=dtype, device=DEV)
+        view = buf[offset:offset + n * ld].view(n, ld)[:, :d]
+        view.copy_(src.to(DEV))
+        return view, buf
+
+    for variant in _variants(n):
+        for k in range(max(_tau(n), 1) + 1):
+            (X, xb), (Y, yb), (G, gb) = put(x, xy_t), put(y, xy_t), put(g, torch.bfloat16)
+            xs, ys, gs = _wide(X), _wide(Y), _wide(G)        # what the kernel reads, widened exactly
+            want_x, want_y = oracle.step(xs, ys, gs, np.float32(gamma), variant, k)
+            scale = max(np.abs(xs).max(), np.abs(ys).max(), gamma * np.abs(gs).max())
+            (Xo, xob), (Yo, yob) = put(torch.zeros(n, d), xy_t), put(torch.zeros(n, d), xy_t)
+            ceca.ceca_gossip_sgd_step_bf16(X, Y, G, gamma, variant, k, X_out=Xo, Y_out=Yo)
+            assert (np.abs(_wide(Xo) - want_x) <= _bf16_tol(want_x, scale, xy_bf16)).all(), (variant, k)
+            assert (np.abs(_wide(Yo) - want_y) <= _bf16_tol(want_y, scale, xy_bf16)).all(), (variant, k)
+            assert torch.isnan(xob[:offset]).all() and torch.isnan(xob[offset + n * ld:]).all()
+            if ld > d:
+                assert torch.isnan(xob[offset:offset + n * ld].view(n, ld)[:, d:]).all()
+                assert torch.isnan(yob[offset:offset + n * ld].view(n, ld)[:, d:]).all()
+            ceca.ceca_gossip_sgd_step_bf16(X, Y, G, gamma, variant, k)     # in place: the same bits
+            assert torch.equal(X, Xo) and torch.equal(Y, Yo)
+    with pytest.raises(ceca.CecaError):   # the gradient is required in this form
+        ceca.ceca_gossip_sgd_step_bf16(X, Y, None, gamma, ceca.CECA_2P, 0)
+
+
+@pytest.mark.parametrize("xy_bf16", [False, True])
+def test_full_size_step_with_bf16_storage_on_column_windows(xy_bf16):
+    """n = 100, d = 25,557,032, CECA-2P, in place: the launch shape bench.py times for the narrow-storage
+    workloads, checked on column windows that include the first and the last (ragged) columns."""
+    n, d, variant, gamma = 100, 25_557_032, ceca.CECA_2P, 0.1
+    _need_free(int(3.3 * n * d * 4))
+    ld = synth.padded_ld(d)
+    xy_t = torch.bfloat16 if xy_bf16 else torch.float32
+    X32, Y32, G32 = synth.step_inputs(n, d, seed=4, x_std=0.01, g_std=0.01, device=DEV, ld=ld)
+    if xy_bf16:
+        X = torch.empty((n, ld), dtype=xy_t, device=DEV)[:, :d]; X.copy_(X32)
+        Y = torch.empty((n, ld), dtype=xy_t, device=DEV)[:, :d]; Y.copy_(Y32)
+        del X32, Y32
+    else:
+        X, Y = X32, Y32
+    G = torch.empty((n, ld), dtype=torch.bfloat16, device=DEV)[:, :d]
+    wins = _windows(d, 4099, 4, seed=n)
+    for k in range(7):
+        synth.gradient_inputs(n, d, k, g_std=0.01, device=DEV, out=G32)
+        G.copy_(G32)
+        before = [(_wide(X[:, lo:hi]), _wide(Y[:, lo:hi]), _wide(G[:, lo:hi])) for lo, hi in wins]
+        ceca.ceca_gossip_sgd_step_bf16(X, Y, G, gamma, variant, k)
+        for (xs, ys, gs), (lo, hi) in zip(before, wins):
+            want_x, want_y = oracle.step(xs, ys, gs, np.float32(gamma), variant, k)
+            scale = max(np.abs(xs).max(), np.abs(ys).max())
+            assert (np.abs(_wide(X[:, lo:hi]) - want_x) <= _bf16_tol(want_x, scale, xy_bf16)).all(), (k, lo)
+            assert (np.abs(_wide(Y[:, lo:hi]) - want_y) <= _bf16_tol(want_y, scale, xy_bf16)).all(), (k, lo)
+
+
 @pytest.mark.parametrize("fused", [0, 1])
 def test_full_size_consensus_on_column_windows(fused):
     """n = 97 (prime), d = 2^20, rows offset by the agent index, tau = 7 rounds, 2-port."""
