@@ -61,6 +61,8 @@ WORKLOADS = {
     "logreg_grad": dict(kind="logreg", n=63, m=2000, d=4096, variant=2, gamma=0.01),
     # whole iterations (gradient kernel + fused step), one CECA cycle captured in a CUDA graph and replayed
     "logreg_train": dict(kind="train", n=63, m=2000, d=4096, variant=2, gamma=0.01, loss="logistic"),
+    # the same with a global average (tau + 1 fused consensus rounds) after every second cycle, all inside the graph
+    "logreg_train_avg": dict(kind="train", n=63, m=2000, d=4096, variant=2, gamma=0.01, loss="logistic", avg_period=2),
     "logreg_train_small": dict(kind="train", n=5, m=100, d=32, variant=2, gamma=0.05, loss="logistic"),
     "lsq_train": dict(kind="train", n=258, m=50, d=10, variant=1, gamma=0.02, loss="square"),
     # n = 2..128 at d = 4,194,304, both variants where defined: kernel and schedule scaling with n
@@ -475,10 +477,21 @@ def bench_train(args, wl, device, dist):
     X = torch.zeros(n, d, device=device); Y = torch.zeros(n, d, device=device); G = torch.empty(n, d, device=device)
     tau = ceca.ceca_schedule(n, variant, 0, peers=False)[0].tau
 
-    def cycle(k0):
+    period = int(wl.get("avg_period", 0))   # cycles between global averages (0: none)
+    status = torch.zeros(64, dtype=torch.int32, device=device)
+
+    def one_cycle(k0):
         for k in range(k0, k0 + tau):
             grad(X, Y, G, k)
             ceca.ceca_gossip_sgd_step(X, Y, G, gamma, variant, k)
+
+    def cycle(k0):
+        """What one graph replay holds: a CECA cycle, or `period` cycles and a global average."""
+        if not period:
+            return one_cycle(k0)
+        for c in range(period):
+            one_cycle(k0 + c * tau)
+        ceca.ceca_consensus_rounds(X, Y, variant, k0 + period * tau, tau + 1, 1, workspace=status)
 
     stream = torch.cuda.current_stream()
     e = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
@@ -507,9 +520,11 @@ def bench_train(args, wl, device, dist):
     torch.cuda.synchronize()
     clocks = sampler.stop()
     graph_ms = e[2].elapsed_time(e[3])
-    iters = args.steps * tau
+    iters = args.steps * tau * max(period, 1)
     peak, which = measured_peak()
     bytes_per_iter = 4 * n * m * d + 8 * n * d + 4 * n * m + (20 * tau - 4) / tau * n * d
+    if period:
+        bytes_per_iter += 16 * n * d / (period * tau)   # the fused average: X, Y in and out
     achieved = bytes_per_iter * iters / (graph_ms * 1e-3) / 1e9
     roof = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak, "traffic": None,
             "kernel": "gradient kernels + step_walk_kernel, whole iteration", "peak_source": "of " + which,
@@ -517,7 +532,10 @@ def bench_train(args, wl, device, dist):
     extra = {"tau": tau, "m": m, "loss": wl["loss"], "iterations_timed": iters, "units": n * d * iters,
              "eager_us_per_iteration": round(eager_ms / iters * 1e3, 2), "graph_us_per_iteration": round(graph_ms / iters * 1e3, 2),
              "l2": "A is %.1f MB" % (n * m * d * 4 / 1e6)}
-    launches = iters * (3 if (d % 4 == 0) else 3)
+    launches = iters * 3 + (args.steps if period else 0)
+    if period:
+        extra["average_every_cycles"] = period
+        assert ceca.ceca_read_status(status) == 0
     return graph_ms, launches, roof, clocks, extra
 
 

@@ -196,6 +196,30 @@ ceca_status_t dsgd_lsq_grad(const float *A, const float *B, const float *X, cons
                             ceca_variant_t variant, void *workspace, size_t workspace_bytes, void *stream);
 
 /*
+ * The gradient for a COLUMN SHARD (not in the paper, whose agents each own a whole model; this is the
+ * form a deployment that splits the d parameter columns over several GPUs needs -- the gossip update
+ * mixes rows only and needs no exchange between column blocks, the gradient needs one):
+ *   1. dsgd_grad_shard_dots   dots[i, s] = <A_i[s, c0:c0+w], z_i[c0:c0+w]>        on every shard
+ *   2. the sum of `dots` over the shards: an all-reduce of n x m floats between GPUs, or
+ *      dsgd_grad_shard_sum (total = part when `first`, else total += part) called shard by shard
+ *      where the shards share a GPU; a fixed order of additions makes the result reproducible
+ *   3. dsgd_grad_shard_apply  turns the summed dots into the per-sample coefficients IN PLACE
+ *      (loss = 0: -(1/m) l sigma(-l t) with targets = labels in {-1, +1}; loss = 1: t - b with
+ *      targets = the measurements b) and writes G[:, c0:c0+w] = sum_s coef_s A_i[s, c0:c0+w] (+ noise)
+ * A_shard: device, n x m x w with row stride lda >= w elements (lda = d when the shard is a view
+ * of the full A, lda = w when it is stored on its own); Z_shard, G_shard, noise_shard: device,
+ * n x w with leading dimensions ldz / ldg (the caller passes the block of X or of Y that
+ * ceca_schedule's `payload` selects); dots: device, n x m.  No workspace.  The same error codes
+ * as the other gradient calls.
+ */
+ceca_status_t dsgd_grad_shard_dots(const float *A_shard, const float *Z_shard, float *dots, int32_t n, int32_t m,
+                                   int64_t w, int64_t lda, int64_t ldz, void *stream);
+ceca_status_t dsgd_grad_shard_sum(float *total, const float *part, int64_t count, int32_t first, void *stream);
+ceca_status_t dsgd_grad_shard_apply(const float *A_shard, const float *targets, float *dots, const float *noise_shard,
+                                    float *G_shard, int32_t n, int32_t m, int64_t w, int64_t lda, int64_t ldg,
+                                    int32_t loss, void *stream);
+
+/*
  * dsgd_logreg_grad for callers that cannot provide a workspace because they cannot allocate device
  * memory when the gradient is needed: a plug-in inside an application that owns the device heap,
  * code running where a framework's allocator must not be re-entered, a latency-critical loop that

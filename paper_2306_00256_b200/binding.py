@@ -17,7 +17,8 @@ WS_STEP_HOST = 4
 EXPORTS = ["ceca_schedule", "ceca_gossip_sgd_step", "ceca_consensus_rounds", "dsgd_logreg_grad",
            "ceca_workspace_bytes", "ceca_read_status", "ceca_gossip_sgd_step_host", "ceca_status_string",
            "dsgd_logreg_grad_static", "dsgd_logreg_grad_static_capacity", "dsgd_lsq_grad",
-           "ceca_fused_wait_selftest", "ceca_gossip_sgd_step_bf16"]
+           "ceca_fused_wait_selftest", "ceca_gossip_sgd_step_bf16", "dsgd_grad_shard_dots", "dsgd_grad_shard_sum",
+           "dsgd_grad_shard_apply"]
 
 
 class Round(ctypes.Structure):
@@ -64,6 +65,12 @@ def library():
     lib.dsgd_logreg_grad.restype = ctypes.c_int
     lib.dsgd_lsq_grad.argtypes = [vp, vp, vp, vp, vp, i64, vp, i32, i32, i64, i64, i32, vp, ctypes.c_size_t, vp]
     lib.dsgd_lsq_grad.restype = ctypes.c_int
+    lib.dsgd_grad_shard_dots.argtypes = [vp, vp, vp, i32, i32, i64, i64, i64, vp]
+    lib.dsgd_grad_shard_dots.restype = ctypes.c_int
+    lib.dsgd_grad_shard_sum.argtypes = [vp, vp, i64, i32, vp]
+    lib.dsgd_grad_shard_sum.restype = ctypes.c_int
+    lib.dsgd_grad_shard_apply.argtypes = [vp, vp, vp, vp, vp, i32, i32, i64, i64, i64, i32, vp]
+    lib.dsgd_grad_shard_apply.restype = ctypes.c_int
     lib.dsgd_logreg_grad_static.argtypes = [vp, vp, vp, vp, i64, vp, i32, i32, i64, i64, i32, vp]
     lib.dsgd_logreg_grad_static.restype = ctypes.c_int
     lib.dsgd_logreg_grad_static_capacity.argtypes = []
@@ -240,6 +247,65 @@ def dsgd_lsq_grad(A, B, X, Y, k, variant, G, workspace, noise=None, stream=None)
                                  _ptr(workspace), ws_bytes, _stream(stream))
     _check(st, "dsgd_lsq_grad")
     return G
+
+
+def shard_columns(d, shards, index, multiple=4):
+    """[c0, c1): the columns of shard `index` when d columns are cut into `shards` contiguous blocks whose
+    boundaries are multiples of `multiple` (so that every block keeps vector alignment); the last block
+    takes the remainder.  Integers only."""
+    if not (0 <= index < shards) or d < 1 or multiple < 1:
+        raise ValueError("bad shard request")
+    units = (d + multiple - 1) // multiple
+    lo = (units * index // shards) * multiple
+    hi = d if index == shards - 1 else (units * (index + 1) // shards) * multiple
+    return min(lo, d), min(hi, d)
+
+
+def _shard3(A, name):
+    """(n, m, w, lda) of a 3-D float32 device tensor whose last dimension is contiguous and whose first two
+    dimensions are laid out as n*m rows of one stride (a column slice of a dense n x m x d tensor is)."""
+    import torch
+    if A.dtype != torch.float32 or A.dim() != 3 or not A.is_cuda or A.stride(2) != 1:
+        raise ValueError("%s must be a 3-D float32 device tensor with unit column stride" % name)
+    n, m, w = A.shape
+    lda = A.stride(1)
+    if m > 1 and n > 1 and A.stride(0) != m * lda:
+        raise ValueError("%s: the sample rows of all agents must be equally spaced" % name)
+    return n, m, w, lda
+
+
+def dsgd_grad_shard_dots(A_shard, Z_shard, dots, stream=None):
+    """dots[i, s] = <A_shard[i, s, :], Z_shard[i, :]> for one column shard."""
+    n, m, w, lda = _shard3(A_shard, "A_shard")
+    _, wz, ldz = _matrix(Z_shard, "Z_shard", n)
+    if wz != w or tuple(dots.shape) != (n, m) or not dots.is_contiguous():
+        raise ValueError("Z_shard must be [n, w] and dots a contiguous [n, m] tensor")
+    st = library().dsgd_grad_shard_dots(_ptr(A_shard), _ptr(Z_shard), _ptr(dots), n, m, w, lda, ldz, _stream(stream))
+    _check(st, "dsgd_grad_shard_dots")
+    return dots
+
+
+def dsgd_grad_shard_sum(total, part, first, stream=None):
+    """total = part (first) or total += part: the sum over shards that share a GPU, in the caller's order."""
+    if total.shape != part.shape or not total.is_contiguous() or not part.is_contiguous():
+        raise ValueError("total and part must be contiguous tensors of one shape")
+    st = library().dsgd_grad_shard_sum(_ptr(total), _ptr(part), total.numel(), int(bool(first)), _stream(stream))
+    _check(st, "dsgd_grad_shard_sum")
+    return total
+
+
+def dsgd_grad_shard_apply(A_shard, targets, dots, G_shard, loss=0, noise_shard=None, stream=None):
+    """Turns the summed dots into coefficients in place and writes the shard's columns of the gradient."""
+    n, m, w, lda = _shard3(A_shard, "A_shard")
+    _, wg, ldg = _matrix(G_shard, "G_shard", n)
+    if wg != w or tuple(dots.shape) != (n, m) or tuple(targets.shape) != (n, m) or not targets.is_contiguous():
+        raise ValueError("G_shard must be [n, w], dots and targets contiguous [n, m] tensors")
+    if noise_shard is not None and _matrix(noise_shard, "noise_shard", n) != (n, w, ldg):
+        raise ValueError("noise_shard must have the shape and row stride of G_shard")
+    st = library().dsgd_grad_shard_apply(_ptr(A_shard), _ptr(targets), _ptr(dots), _ptr(noise_shard), _ptr(G_shard),
+                                         n, m, w, lda, ldg, int(loss), _stream(stream))
+    _check(st, "dsgd_grad_shard_apply")
+    return G_shard
 
 
 def dsgd_logreg_grad_static(A, labels, X, Y, k, variant, G, stream=None):

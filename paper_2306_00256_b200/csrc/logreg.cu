@@ -282,6 +282,103 @@ extern "C" ceca_status_t dsgd_lsq_grad(const float *A, const float *B, const flo
   return enqueue_grad<kLossSquare>(A, B, Z, noise, G, n, m, d, ld, workspace, static_cast<cudaStream_t>(stream));
 }
 
+// ---- column-sharded form -----------------------------------------------------------------------
+//
+// When the parameter columns are split over several GPUs (the update itself mixes rows only, so a
+// column block needs no exchange for it), a shard holds A[:, :, c0:c0+w] and z[:, c0:c0+w] and the
+// gradient splits into (i) the partial inner products of the block, (ii) their sum over the shards
+// (n x m floats: the one exchange per iteration, an all-reduce between GPUs) and (iii) the
+// coefficient per sample and the block's share of A^T coef.  A is read once in (i) and once in (iii).
+namespace ceca {
+
+__global__ void __launch_bounds__(256) shard_dots_kernel(const float *A, const float *Z, float *dots, int32_t n,
+                                                         int32_t m, int64_t w, int64_t lda, int64_t ldz, int vec) {
+  const int64_t sample = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;  // one warp per sample
+  const int lane = threadIdx.x & 31;
+  if (sample >= (int64_t)n * m) return;
+  const int64_t i = sample / m;
+  const float *row = A + sample * lda;
+  const float *z = Z + i * ldz;
+  float t = 0.f;
+  if (vec) {
+    for (int64_t c = 4 * lane; c < w; c += 128)
+      t += dot4(__ldcs(reinterpret_cast<const float4 *>(row + c)), *reinterpret_cast<const float4 *>(z + c));
+  } else {
+    for (int64_t c = lane; c < w; c += 32) t = fmaf(row[c], z[c], t);
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
+  if (lane == 0) dots[sample] = t;
+}
+
+__global__ void __launch_bounds__(256) shard_sum_kernel(float *total, const float *part, int64_t count, int first) {
+  const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx < count) total[idx] = first ? part[idx] : total[idx] + part[idx];
+}
+
+template <int LOSS>
+__global__ void __launch_bounds__(256) shard_coef_kernel(float *dots, const float *targets, int64_t count, float inv_m) {
+  const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx < count) dots[idx] = sample_coef<LOSS>(targets[idx], dots[idx], inv_m);
+}
+
+__global__ void __launch_bounds__(256) shard_accum_kernel(const float *A, const float *coef, const float *noise,
+                                                          float *G, int32_t n, int32_t m, int64_t w, int64_t lda,
+                                                          int64_t ldg) {
+  const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= (int64_t)n * w) return;
+  const int64_t i = idx / w, c = idx - i * w;
+  const float *col = A + i * m * lda + c;
+  const float *cf = coef + i * m;
+  float g = 0.f;
+  for (int32_t s = 0; s < m; ++s) g = fmaf(cf[s], col[(int64_t)s * lda], g);
+  if (noise) g += noise[i * ldg + c];
+  G[i * ldg + c] = g;
+}
+
+}  // namespace ceca
+
+extern "C" ceca_status_t dsgd_grad_shard_dots(const float *A_shard, const float *Z_shard, float *dots, int32_t n,
+                                              int32_t m, int64_t w, int64_t lda, int64_t ldz, void *stream) {
+  using namespace ceca;
+  if (!A_shard || !Z_shard || !dots || n < 1 || m < 1 || w < 1 || lda < w || ldz < w) return CECA_ERR_INVALID_ARG;
+  const int64_t blocks = ((int64_t)n * m * 32 + 255) / 256;
+  if (blocks > 0x7fffffffLL) return CECA_ERR_UNSUPPORTED;
+  const int vec = (w % 4 == 0) && (lda % 4 == 0) && (ldz % 4 == 0) && aligned16(A_shard) && aligned16(Z_shard);
+  shard_dots_kernel<<<(unsigned)blocks, 256, 0, static_cast<cudaStream_t>(stream)>>>(A_shard, Z_shard, dots, n, m, w,
+                                                                                      lda, ldz, vec);
+  return cudaGetLastError() == cudaSuccess ? CECA_OK : CECA_ERR_CUDA;
+}
+
+extern "C" ceca_status_t dsgd_grad_shard_sum(float *total, const float *part, int64_t count, int32_t first,
+                                             void *stream) {
+  using namespace ceca;
+  if (!total || !part || count < 1) return CECA_ERR_INVALID_ARG;
+  const int64_t blocks = (count + 255) / 256;
+  if (blocks > 0x7fffffffLL) return CECA_ERR_UNSUPPORTED;
+  shard_sum_kernel<<<(unsigned)blocks, 256, 0, static_cast<cudaStream_t>(stream)>>>(total, part, count, first != 0);
+  return cudaGetLastError() == cudaSuccess ? CECA_OK : CECA_ERR_CUDA;
+}
+
+extern "C" ceca_status_t dsgd_grad_shard_apply(const float *A_shard, const float *targets, float *dots,
+                                               const float *noise_shard, float *G_shard, int32_t n, int32_t m,
+                                               int64_t w, int64_t lda, int64_t ldg, int32_t loss, void *stream) {
+  using namespace ceca;
+  if (!A_shard || !targets || !dots || !G_shard || n < 1 || m < 1 || w < 1 || lda < w || ldg < w)
+    return CECA_ERR_INVALID_ARG;
+  if (loss != kLossLogistic && loss != kLossSquare) return CECA_ERR_INVALID_ARG;
+  const int64_t count = (int64_t)n * m;
+  const int64_t blocks1 = (count + 255) / 256, blocks2 = ((int64_t)n * w + 255) / 256;
+  if (blocks1 > 0x7fffffffLL || blocks2 > 0x7fffffffLL) return CECA_ERR_UNSUPPORTED;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const float inv_m = (float)(1.0 / (double)m);
+  if (loss == kLossLogistic) shard_coef_kernel<kLossLogistic><<<(unsigned)blocks1, 256, 0, s>>>(dots, targets, count, inv_m);
+  else shard_coef_kernel<kLossSquare><<<(unsigned)blocks1, 256, 0, s>>>(dots, targets, count, inv_m);
+  if (cudaGetLastError() != cudaSuccess) return CECA_ERR_CUDA;
+  shard_accum_kernel<<<(unsigned)blocks2, 256, 0, s>>>(A_shard, dots, noise_shard, G_shard, n, m, w, lda, ldg);
+  return cudaGetLastError() == cudaSuccess ? CECA_OK : CECA_ERR_CUDA;
+}
+
 // ---- the same gradient for callers that cannot hand over a workspace ---------------------------
 //
 // Some callers have no way to get device memory at the moment they need the gradient: a plug-in

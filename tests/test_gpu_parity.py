@@ -598,6 +598,45 @@ def test_small_logistic_regression_run(n, variant):
 # least-squares gradient and the paper's convex experiment (Sec. 5 "DSGD: least-squares problem")
 # --------------------------------------------------------------------------------------------
 
+@pytest.mark.parametrize("shards", [1, 2, 3])
+@pytest.mark.parametrize("n,m,d,view", [(5, 100, 32, True), (6, 37, 1030, True), (3, 50, 4099, False), (63, 40, 512, False)])
+def test_column_sharded_logistic_gradient(shards, n, m, d, view):
+    """The gradient computed shard by shard (partial dot products per column block, their sum in shard order,
+    coefficient + A^T pass per block) equals the oracle's and the unsharded kernel's; unequal block widths."""
+    a, lab, _ = synth.logreg_problem(n, m, d, seed=n + d, flip=0.1, hetero_std=0.5)
+    gen = torch.Generator().manual_seed(d)
+    x, y = 0.1 * torch.randn(n, d, generator=gen), 0.1 * torch.randn(n, d, generator=gen)
+    A, L, X, Y = a.to(DEV), lab.to(DEV), x.to(DEV), y.to(DEV)
+    ws = torch.empty(ceca.ceca_workspace_bytes(ceca.WS_LOGREG_GRAD, n, m, d), dtype=torch.uint8, device=DEV)
+    for k in (0, 1, 2):
+        variant = ceca.CECA_2P
+        Z = Y if ceca.ceca_schedule(n, variant, k, peers=False)[0].payload else X
+        want = oracle.logreg_grad(_np(a), _np(lab), _np(x), _np(y), k)
+        whole = torch.empty(n, d, device=DEV)
+        ceca.dsgd_logreg_grad(A, L, X, Y, k, variant, whole, ws)
+        G = torch.full((n, d), float("nan"), device=DEV)
+        cuts = [ceca.shard_columns(d, shards, j) for j in range(shards)]
+        assert cuts[0][0] == 0 and cuts[-1][1] == d and all(cuts[j][1] == cuts[j + 1][0] for j in range(shards - 1))
+        total, part = torch.empty(n, m, device=DEV), torch.empty(n, m, device=DEV)
+        blocks = []
+        for j, (lo, hi) in enumerate(cuts):
+            # a shard either views its columns of the full matrices or owns a dense copy of them
+            As = A[:, :, lo:hi] if view else A[:, :, lo:hi].contiguous()
+            Zs = Z[:, lo:hi] if view else Z[:, lo:hi].contiguous()
+            blocks.append(As)
+            ceca.dsgd_grad_shard_dots(As, Zs, part)
+            ceca.dsgd_grad_shard_sum(total, part, first=(j == 0))
+        for j, (lo, hi) in enumerate(cuts):
+            dots = total.clone()          # every shard gets its own copy of the summed dots: apply overwrites it
+            Gs = G[:, lo:hi] if view else torch.empty(n, hi - lo, device=DEV)
+            ceca.dsgd_grad_shard_apply(blocks[j], L, dots, Gs)
+            if not view:
+                G[:, lo:hi] = Gs
+        tol = _grad_tol(d, want)
+        assert np.abs(_np(G) - want).max() <= tol, (k, shards)
+        assert np.abs(_np(G) - _np(whole)).max() <= tol, (k, shards)
+
+
 def _lsq_tol(a, b, z):
     """fp32 bound: a length-d dot product per residual, then a length-m sum of residual * feature."""
     n, m, d = a.shape
@@ -723,6 +762,61 @@ def test_full_size_step_on_column_windows(n, d, variant, iters):
             # and the whole trajectory against an fp64 run from the same start
             ref[w] = oracle.step(ref[w][0], ref[w][1], gw[w], np.float32(gamma), variant, k)
             assert np.abs(_np(X[:, lo:hi]) - ref[w][0]).max() <= tol * (k + 1)
+
+
+def test_device_entry_points_reject_bad_arguments_and_launch_nothing():
+    """The argument-error table of the C ABI with real device buffers: every call must come back with the
+    stated status before anything is enqueued, so the NaN-filled outputs stay untouched."""
+    import ctypes
+    lib = ceca.library()
+    big = 2050 * 8
+    bufs = [torch.full((big + 4,), float("nan"), device=DEV) for _ in range(6)]
+    x, y, g, xo, yo, ws = [ctypes.c_void_p(b.data_ptr()) for b in bufs]
+    xo_off = ctypes.c_void_p(bufs[3].data_ptr() + 4)     # 4 bytes past a 16-byte boundary
+    stream = ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+    step = lib.ceca_gossip_sgd_step
+    assert step(None, y, g, xo, yo, 4, 8, 8, 0.1, 2, 0, stream) == 1
+    assert step(x, y, g, xo, yo, 0, 8, 8, 0.1, 2, 0, stream) == 1
+    assert step(x, y, g, xo, yo, 4, 8, 7, 0.1, 2, 0, stream) == 1        # ld < d
+    assert step(x, y, g, xo, yo, 5, 8, 8, 0.1, 1, 0, stream) == 2        # odd n, 1-port
+    assert step(x, None, g, xo, yo, 4, 8, 8, 0.1, 2, 1, stream) == 1     # round 1 needs Y
+    assert step(x, y, g, xo, xo, 4, 8, 8, 0.1, 2, 1, stream) == 4        # X_out == Y_out
+    assert step(x, y, g, y, yo, 4, 8, 8, 0.1, 2, 1, stream) == 4         # X_out == Y
+    assert step(x, None, g, xo, None, 6, 8, 8, 0.1, 2, 0, stream) == 1   # X-only needs n = 2^tau
+    assert step(x, y, g, xo, None, 8, 8, 8, 0.1, 2, 0, stream) == 1      # y+ may only be dropped at r = tau-1
+    assert step(x, y, g, xo, yo, 4, 8, 8, 0.1, 3, 0, stream) == 1        # no such variant
+    assert step(x, y, g, xo, yo, 4, 8, 8, 0.1, 2, -1, stream) == 1       # k < 0
+    bf = lib.ceca_gossip_sgd_step_bf16
+    assert bf(x, y, None, xo, yo, 4, 8, 8, 0, 0.1, 2, 0, stream) == 1    # the narrow gradient is required
+    assert bf(x, y, g, xo, None, 4, 8, 8, 1, 0.1, 2, 0, stream) == 1     # so is Y_out
+    assert bf(x, y, g, g, yo, 4, 8, 8, 1, 0.1, 2, 0, stream) == 4        # X_out == G
+    cons = lib.ceca_consensus_rounds
+    assert cons(x, y, xo, yo, 4, 8, 8, 2, 0, -1, 0, None, 0, stream) == 1
+    assert cons(x, None, xo, None, 6, 8, 8, 2, 0, 2, 0, None, 0, stream) == 5      # no Y_out, no workspace (n not 2^tau)
+    assert cons(x, None, xo, None, 2050, 8, 8, 2, 0, 2, 1, ws, 256, stream) == 4   # n > 2048 fused
+    assert cons(x, None, xo, None, 200, 8, 8, 2, 0, 2, 3, ws, 256, stream) == 4    # tensor-memory kernel: n <= 128
+    assert cons(x, None, xo, None, 6, 8, 8, 1, 0, 2, 4, ws, 256, stream) == 4      # register-block kernel: 2-port only
+    assert cons(x, None, xo, None, 4, 8, 8, 2, 0, 2, 7, ws, 256, stream) == 1      # no such kernel
+    assert cons(x, None, xo_off, None, 4, 8, 8, 2, 0, 2, 1, ws, 256, stream) == 3  # misaligned
+    assert cons(x, None, xo, None, 4, 8, 6, 2, 0, 2, 1, ws, 256, stream) == 1      # ld < d
+    assert cons(x, None, xo, None, 4, 6, 6, 2, 0, 2, 1, ws, 256, stream) == 3      # ld*4 % 16
+    assert cons(x, None, xo, None, 4, 8, 8, 2, 1, 2, 1, ws, 256, stream) == 1      # starts at r=1, no Y
+    assert cons(x, None, xo, None, 4, 8, 8, 2, 0, 2, 1, None, 0, stream) == 5      # fused needs the status word
+    assert cons(x, None, xo, yo, 4, 8, 8, 2, 3, 0, 1, ws, 256, stream) == 1        # zero rounds, Y_out without Y
+    self_test = lib.ceca_fused_wait_selftest
+    assert self_test(x, x, 6, 32, 32, 2, ws, 256, stream) == 4                     # X_out must not alias X
+    assert self_test(x, xo, 6, 32, 32, 1, ws, 256, stream) == 1                    # names a kernel, not "auto"
+    grad = lib.dsgd_logreg_grad
+    assert grad(x, y, g, g, 0, xo, 4, 0, 8, 8, 2, ws, 1 << 10, stream) == 1
+    assert grad(x, y, g, g, 0, xo, 4, 5, 8, 8, 2, None, 0, stream) == 5
+    assert grad(x, y, g, None, 1, xo, 6, 5, 8, 8, 2, ws, 1 << 10, stream) == 1     # n=6, k=1 evaluates at Y
+    assert lib.dsgd_logreg_grad_static(x, y, g, None, 1, xo, 6, 5, 8, 8, 2, stream) == 1
+    host = lib.ceca_gossip_sgd_step_host
+    assert host(x, y, g, 4, 8, 8, 0.1, 2, 0, None, 0) == 5
+    assert host(x, y, g, 5, 8, 8, 0.1, 1, 0, ws, 1 << 10) == 2
+    torch.cuda.synchronize()
+    for b in bufs:
+        assert torch.isnan(b).all()
 
 
 # --------------------------------------------------------------------------------------------

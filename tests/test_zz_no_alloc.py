@@ -44,10 +44,16 @@ def test_static_scratch_gradient_matches_workspace_gradient_on_consecutive_calls
         ws = torch.empty(ceca.ceca_workspace_bytes(ceca.WS_LOGREG_GRAD, n, m, d), dtype=torch.uint8, device=DEV)
         want_gpu = torch.full((n, d), float("nan"), device=DEV)
         ceca.dsgd_logreg_grad(A, L, X, Y, k, variant, want_gpu, ws)
-        for _ in range(2):   # twice in a row on the same inputs as well
+        for call in range(2):   # twice in a row on the same inputs as well
             got = torch.full((n, d), float("nan"), device=DEV)
+            torch.cuda.synchronize()
+            free_before = torch.cuda.mem_get_info()[0]
             ceca.dsgd_logreg_grad_static(A, L, X, Y, k, variant, got)
             torch.cuda.synchronize()
+            if call == 1 or (n, m, d) != cases[0][:3]:
+                # the property in the name: the device has exactly as much free memory after the call as
+                # before it (the very first call of a process may still load the kernels' module lazily)
+                assert torch.cuda.mem_get_info()[0] == free_before
             want = oracle.logreg_grad(a.numpy(), lab.numpy(), x.numpy(), y.numpy(), k)
             assert np.abs(got.cpu().numpy() - want_gpu.cpu().numpy()).max() <= _tol(d, want)
             assert np.abs(got.cpu().numpy() - want).max() <= _tol(d, want)
