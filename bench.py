@@ -47,16 +47,18 @@ WORKLOADS = {
     "step_small": dict(kind="step", n=100, d=2_097_152, variant=2, gamma=0.1),
     # n a power of two: the X-only update (12 B per agent-parameter; CECA-2P = one-peer exponential graph)
     "pow2_xonly_step": dict(kind="step", n=128, d=8_388_608, variant=2, gamma=0.1, x_only=True),
-    # fused = 1 picks the kernel by n (tensor-memory exchange up to n = 128, shared-memory exchange above)
+    # fused = 1 picks the kernel by n and variant (register blocks for CECA-2P up to n = 1152, shared-memory exchange otherwise)
     "consensus_fused": dict(kind="consensus", n=97, d=1 << 20, variant=2, fused=1),
     "consensus_fused_smem": dict(kind="consensus", n=97, d=1 << 20, variant=2, fused=2),
     "consensus_fused_tmem": dict(kind="consensus", n=97, d=1 << 20, variant=2, fused=3),
     "consensus_rounds": dict(kind="consensus", n=97, d=1 << 20, variant=2, fused=0),
     # half the columns: the case the profiler captures are taken on (0.2 GB in, 0.4 GB out)
     "consensus_fused_small": dict(kind="consensus", n=97, d=1 << 19, variant=2, fused=1),
-    # the paper's network sizes (Sec. 5): n = 130 (32-column tiles) and n = 1026 (8-column tiles, eleven rounds)
+    # the paper's network sizes (Sec. 5): n = 130, n = 258 (32-column tiles) and n = 1026 (16-column tiles, eleven rounds)
     "consensus_fused_130": dict(kind="consensus", n=130, d=1 << 20, variant=2, fused=1),
+    "consensus_fused_258": dict(kind="consensus", n=258, d=1 << 19, variant=2, fused=1),
     "consensus_fused_1026": dict(kind="consensus", n=1026, d=1 << 18, variant=2, fused=1),
+    "consensus_fused_1026_smem": dict(kind="consensus", n=1026, d=1 << 18, variant=2, fused=2),
     "consensus_rounds_1026": dict(kind="consensus", n=1026, d=1 << 18, variant=2, fused=0),
     "logreg_grad": dict(kind="logreg", n=63, m=2000, d=4096, variant=2, gamma=0.01),
     # whole iterations (gradient kernel + fused step), one CECA cycle captured in a CUDA graph and replayed
@@ -410,7 +412,7 @@ def bench_consensus(args, wl, device, dist):
         kernel = "step_walk_kernel<float4, no gradient> x tau"
     elif fused == 3:
         kernel = "consensus_tmem_kernel (tensor-memory exchange)"
-    elif fused == 2 or n > 256 or variant != 2:
+    elif fused == 2 or n > 1152 or variant != 2:
         kernel = "consensus_fused_kernel (shared-memory exchange of every row)"
     else:
         kernel = "consensus_block_kernel (register blocks, boundary rows through shared memory)"
@@ -588,13 +590,13 @@ def bench_sweep(args, wl, device, dist):
                                                "l2": "n >= 8 rows of 16.8 MB per array exceed L2; smaller n partly L2-resident"}
 
 
-SECONDARY = ["consensus_fused", "consensus_rounds", "consensus_fused_130", "consensus_fused_1026", "logreg_grad",
-             "resnet18_step"]
+SECONDARY = ["consensus_fused", "consensus_rounds", "consensus_fused_130", "consensus_fused_258", "consensus_fused_1026",
+             "logreg_grad", "resnet18_step"]
 
 
 def run_secondary(device, steps=20, warmup=5):
     """Short legs of the other configurations, attached to the default line as `secondary`: the fused and the
-    per-round consensus at n = 97, the fused consensus at the paper's n = 130 and n = 1026, the logistic gradient
+    per-round consensus at n = 97, the fused consensus at the paper's n = 130, 258 and 1026, the logistic gradient
     at n = 63, m = 2000, d = 4096 and the 1-port step at ResNet-18 size.  Each leg is the same function a
     --workload run of that name calls, with its own inputs, warm-up and CUDA events."""
     import torch

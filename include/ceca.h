@@ -139,12 +139,17 @@ ceca_status_t ceca_gossip_sgd_step_bf16(const void *X, const void *Y, const void
  *              without any workspace when n is a power of two (J then never feeds I).
  *   fused = 1 (CECA_FUSED_AUTO): a single launch.  A column tile of all n rows is brought on chip
  *              by TMA (cp.async.bulk.tensor), every round runs there, and the tile is written back
- *              once.  Two kernels exist and 1 picks by n:
- *                2 (CECA_FUSED_SMEM) exchanges the rows through shared memory; n <= 2048 (32-column
- *                  tiles up to n = 256, 8-column tiles above);
- *                3 (CECA_FUSED_TMEM) exchanges them through tensor memory (tcgen05.st / tcgen05.ld)
- *                  and is the faster one where it applies: 2 <= n <= 128.
- *              Passing 2 or 3 forces that kernel (CECA_ERR_UNSUPPORTED outside its range).
+ *              once.  Three kernels exist and 1 picks by n and variant:
+ *                4 (CECA_FUSED_BLOCK) keeps contiguous blocks of agents in registers, so that most of
+ *                  the exchange is register to register and only block boundaries go through shared
+ *                  memory; CECA-2P, 2 <= n <= 1152 (64-column tiles up to n = 256, 32-column tiles up
+ *                  to n = 512, 16-column tiles above).  The fastest one where it applies.
+ *                2 (CECA_FUSED_SMEM) exchanges every row through shared memory; both variants,
+ *                  n <= 2048 (32-column tiles up to n = 256, 8-column tiles above).  What 1 falls back
+ *                  to for CECA-1P and for 1152 < n <= 2048.
+ *                3 (CECA_FUSED_TMEM) exchanges the rows through tensor memory (tcgen05.st /
+ *                  tcgen05.ld); 2 <= n <= 128.  Kept for comparison; never picked by 1.
+ *              Passing 2, 3 or 4 forces that kernel (CECA_ERR_UNSUPPORTED outside its range).
  *              All need X / X_out (and Y / Y_out when used) 16-byte aligned with ld*4 a multiple of
  *              16 (else CECA_ERR_ALIGNMENT), ld < 2^32 (more than 64 rounds run as several
  *              launches and then need Y_out), and a workspace of

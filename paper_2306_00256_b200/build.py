@@ -9,7 +9,7 @@ CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libceca_b200.so")
 
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-              "-Xptxas=-v", "-shared", "-Xcompiler", "-fPIC"]
+              "-Xptxas=-v", "-shared", "-Xcompiler", "-fPIC", "--threads", "8"]
 
 
 def sources():

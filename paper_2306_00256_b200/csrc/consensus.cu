@@ -1,18 +1,19 @@
 // CECA consensus rounds (Sec. 3.1 "Main recursions", Algorithm 2; Sec. 3.2 for the 1-port pairing).
 //
 // fused = 0: one pass of the step kernel (gamma = 0, no G) per round.
-// fused = 1: one launch.  Each CTA brings an n x W column tile of X (and of Y when the first
-//   round needs it) into shared memory with one TMA tensor load, moves it into registers (a
-//   thread keeps a few rows of eight columns for the whole run), and runs all rounds on chip: per
-//   round every thread publishes the payload (I or J) of its rows in a shared exchange buffer,
-//   the CTA synchronises, and every thread picks up the value of the row it receives from.  Only
-//   4 bytes per element per round go through shared memory in each direction (128-bit accesses,
-//   packed two-wide fp32 FMAs; eight columns per thread keep the index arithmetic per element
-//   small).  The finished tiles go back with one TMA tensor store each.  HBM sees X once in and
-//   X (and Y) once out, instead of once per round.  Several CTAs per SM overlap each other's
-//   load, compute and store phases.  Tiles are 32 columns wide for n <= 256 (one TMA box); for
-//   256 < n <= 2048 they are 8 columns wide and made of several boxes, so that all rows still fit
-//   in shared memory.
+// fused = 1: one launch.  Three kernels; this file holds the dispatch and the one that exchanges every
+//   row through shared memory (the register-block kernel and the tensor-memory kernel have files of
+//   their own).  Each CTA brings an n x W column tile of X (and of Y when the first round needs it)
+//   into shared memory with one TMA tensor load, moves it into registers (a thread keeps a few rows
+//   of eight columns for the whole run), and runs all rounds on chip: per round every thread
+//   publishes the payload (I or J) of its rows in a shared exchange buffer, the CTA synchronises,
+//   and every thread picks up the value of the row it receives from.  Only 4 bytes per element per
+//   round go through shared memory in each direction (128-bit accesses, packed two-wide fp32 FMAs;
+//   eight columns per thread keep the index arithmetic per element small).  The finished tiles go
+//   back with one TMA tensor store each.  HBM sees X once in and X (and Y) once out, instead of once
+//   per round.  Several CTAs per SM overlap each other's load, compute and store phases.  Tiles are
+//   32 columns wide for n <= 256 (one TMA box); for 256 < n <= 2048 they are 8 columns wide and made
+//   of several boxes, so that all rows still fit in shared memory.
 #include <cuda.h>
 #include <cuda_runtime.h>
 

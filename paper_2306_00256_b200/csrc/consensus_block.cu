@@ -2,11 +2,19 @@
 // blocks of agents: most of every round's exchange never leaves the register file, and what the
 // kernel executes per value and round is close to the one fused multiply-add it has to do.
 //
-// Layout.  A CTA of P warps owns one 64-column tile of all n rows (TMA tensor load into shared
-// memory).  A lane is two adjacent matrix columns; warp p keeps I and J of a contiguous block of
-// agents (rows i0 .. i0+cnt-1) of those columns in registers, at static register positions.  The
-// block size is a template argument CB = ceil(n / P): the first blocks hold CB agents, the others
-// CB-1, so every loop over a block has a compile-time trip count and at most one predicated row.
+// Layout.  A CTA owns one column tile of all n rows (TMA tensor loads into shared memory).  A thread
+// is two adjacent matrix columns of one block of agents: LPB threads side by side cover the 2 * LPB
+// columns of the tile, and each keeps I and J of a contiguous block of CB agents (rows i0 .. i0+CB-1)
+// of its two columns in registers, at static register positions.  LPB = 32 (a block is a warp, 64-column
+// tiles) serves n <= 256; LPB = 16 and 8 (32- and 16-column tiles, two and four blocks per warp) let
+// all rows of a tile fit on one SM up to n = 512 and n = 1152 (the paper's n = 1026).  Two ways of
+// cutting n rows into blocks, both with compile-time trip counts for every loop over a block:
+//   balanced (LPB >= 16): the first blocks hold CB agents, the others CB-1 (one predicated row);
+//   uniform (LPB = 8): every block holds CB agents except the last, which holds what is left; its
+//     surplus register rows ("phantom" rows, index >= n) are computed like the others but never
+//     stored, and no real row ever receives from one, because sources are taken modulo n.  Threads
+//     beyond the last block duplicate it (same values to the same shared-memory addresses) and
+//     store nothing.  Equal block sizes are what keeps the 16-column tiles free of bank conflicts.
 //
 // Why this cuts the exchange.  In round r of CECA-2P agent i receives from agent i - s with
 // s = n_r + delta_r, and s roughly doubles every round (1, 2, 3, 6, 12, 24, 48 for n = 97).  While
@@ -14,10 +22,11 @@
 // thread: a register-to-register update with compile-time indices (one instantiation of the round
 // body per value of s, selected by a uniform switch).  Only the first s rows of a block need a
 // value from the previous block, so only the last s rows of every block are published in shared
-// memory.  Rounds with s >= block size exchange every row.  For n = 97 (blocks of 12-13 agents)
-// that is (1+2+3+6+12)/13 + 2 = 3.9 full exchanges instead of 7.  All shared-memory accesses are
-// 64-bit and conflict free (a warp touches 64 consecutive floats of one row), addressed as one
-// base pointer plus compile-time offsets.
+// memory.  Rounds with s >= block size exchange every row.  For n = 97 (blocks of 25 agents)
+// that is (1+2+3+6+12+24)/25 + 1 = 2.9 full exchanges instead of 7.  All shared-memory accesses are
+// 64-bit, addressed as one base pointer plus compile-time offsets, and conflict free: half a warp
+// touches 32 consecutive floats of one row (LPB >= 16), or, for LPB = 8, two 16-float row segments
+// that lie CB rows apart -- CB is odd there, so the two fall into different halves of the 32 banks.
 //
 // Pipeline.  CTAs are persistent.  The first round reads the neighbours' payload straight from the
 // landed tile (it holds exactly the not-yet-updated values), so it publishes nothing and needs no
@@ -49,10 +58,9 @@
 
 namespace ceca {
 
-constexpr int kBkTileCols = 64;
 constexpr int kBkMaxRounds = 64;
 constexpr int kBkRenormEvery = 16;
-constexpr int kBkMaxCb = 25;            // agents per block (100 state registers)
+constexpr int kBkMaxBoxRows = 256;      // a TMA box holds at most 256 rows; taller tiles land as several boxes
 constexpr uint32_t kBkWaitPolls = 1u << 22;
 
 constexpr int kBkPayloadJ = 1;  // the message is J (else I)
@@ -72,7 +80,11 @@ struct BlockArgs {
   float *Xo, *Yo;
   int64_t ld;
   int32_t d, n, rounds, has_y_in, has_y_out, tiles;
-  int32_t nfull;       // blocks 0..nfull-1 hold CB agents, the others CB-1
+  int32_t blocks;      // blocks of agents
+  int32_t nfull;       // balanced: blocks 0 .. nfull-1 hold CB agents, the others CB-1;
+                       // uniform: blocks 0 .. nfull-1 (= blocks-1 or blocks) hold CB, the last one the rest
+  int32_t boxes, box_rows;   // a tile lands as `boxes` TMA boxes of `box_rows` rows (boxes * box_rows >= n)
+  uint32_t tile_bytes; // shared-memory footprint of one tile (a multiple of 128 that holds blocks * CB rows and all boxes)
   int32_t single_xch;  // one exchange tile instead of two (saves shared memory, costs a second barrier per round)
   int32_t wait_polls;
   uint32_t tx_bytes;   // bytes the landing barrier is armed for
@@ -113,8 +125,7 @@ __device__ __forceinline__ void static_for(F &&f) {
 #define CECA_IDX(I) decltype(I)::value
 
 // Shared memory is addressed by 32-bit shared-window addresses with compile-time byte offsets, so
-// that an access costs one instruction and no address arithmetic.
-constexpr int kBkRowBytes = kBkTileCols * (int)sizeof(float);
+// that an access costs one instruction and no address arithmetic.  RB = bytes per tile row.
 template <int OFF>
 __device__ __forceinline__ pk2 lds64(uint32_t addr) {
   pk2 v;
@@ -132,20 +143,25 @@ struct BlockPos {
   uint32_t own;    // row i0 of the exchange tile
   uint32_t prev;   // in-register rounds: the row just after the S source rows (row i0; row n for block 0)
   uint32_t col;    // row 0
-  int i0, cnt, n;
-  bool full_block, publish;
+  int i0, cnt;     // cnt = real rows of the block (CB, fewer in the last block)
+  bool full, publish;
 };
 
-// One round with a compile-time shift S smaller than every block.  Z (the payload) is Ih or Jh itself.
-template <int CB, int S, bool PAYJ>
+// One round with a compile-time shift S smaller than a block.  Z (the payload) is Ih or Jh itself.
+template <int CB, int RB, bool BAL, int CH, int S, bool PAYJ>
 __device__ __forceinline__ void round_partial(pk2 (&Ih)[CB], pk2 (&Jh)[CB], pk2 cI, pk2 cJ, const BlockPos &q) {
   pk2(&Z)[CB] = PAYJ ? Jh : Ih;
   if (q.publish) {
-    // the last S rows of the block are what the next block's first S rows receive
-    if (q.full_block) {
-      static_for<S>([&](auto T) { sts64<(CB - S + CECA_IDX(T)) * kBkRowBytes>(q.own, Z[CB - S + CECA_IDX(T)]); });
-    } else if constexpr (CB - 1 - S >= 0) {
-      static_for<S>([&](auto T) { sts64<(CB - 1 - S + CECA_IDX(T)) * kBkRowBytes>(q.own, Z[CB - 1 - S + CECA_IDX(T)]); });
+    // the last S rows of a block are what the next block's first S rows receive
+    if (q.full) {
+      static_for<S>([&](auto T) { sts64<(CB - S + CECA_IDX(T)) * RB>(q.own, Z[CB - S + CECA_IDX(T)]); });
+    } else if constexpr (BAL) {   // a block of CB - 1 rows
+      if constexpr (CB - 1 - S >= 0)
+        static_for<S>([&](auto T) { sts64<(CB - 1 - S + CECA_IDX(T)) * RB>(q.own, Z[CB - 1 - S + CECA_IDX(T)]); });
+    } else {
+      // the last block of the uniform cut publishes all its rows, wherever its real ones end
+      // (block 0 finds them just below row n)
+      static_for<CB>([&](auto J) { sts64<CECA_IDX(J) * RB>(q.own, Z[CECA_IDX(J)]); });
     }
     __syncthreads();
   }
@@ -155,13 +171,13 @@ __device__ __forceinline__ void round_partial(pk2 (&Ih)[CB], pk2 (&Jh)[CB], pk2 
     Ih[j] = axpy2(cI, z, Ih[j]);
     Jh[j] = axpy2(cJ, z, Jh[j]);
   }
-  // the first S rows receive from the S rows before the block (no wrap inside), eight loads in flight at a time
-  constexpr int kChunk = 8;
+  // the first S rows receive from the S rows before the block (no wrap inside), CH loads in flight at a time
+  constexpr int kChunk = CH;
   static_for<(S + kChunk - 1) / kChunk>([&](auto C) {
     constexpr int T0 = CECA_IDX(C) * kChunk;
     constexpr int TN = S - T0 < kChunk ? S - T0 : kChunk;
     pk2 R[TN];
-    static_for<TN>([&](auto T) { R[CECA_IDX(T)] = lds64<(T0 + CECA_IDX(T) - S) * kBkRowBytes>(q.prev); });
+    static_for<TN>([&](auto T) { R[CECA_IDX(T)] = lds64<(T0 + CECA_IDX(T) - S) * RB>(q.prev); });
     static_for<TN>([&](auto T) {
       Ih[T0 + CECA_IDX(T)] = axpy2(cI, R[CECA_IDX(T)], Ih[T0 + CECA_IDX(T)]);
       Jh[T0 + CECA_IDX(T)] = axpy2(cJ, R[CECA_IDX(T)], Jh[T0 + CECA_IDX(T)]);
@@ -170,26 +186,28 @@ __device__ __forceinline__ void round_partial(pk2 (&Ih)[CB], pk2 (&Jh)[CB], pk2 
 }
 
 // One round in which every row receives through shared memory (s at least as large as a block).
-template <int CB, bool PAYJ>
-__device__ __forceinline__ void round_full(pk2 (&Ih)[CB], pk2 (&Jh)[CB], pk2 cI, pk2 cJ, const BlockPos &q, int s) {
+// Uniform cut: phantom rows are published and updated like real ones; their addresses stay inside
+// the tile (it holds blocks * CB rows), and what they receive is never used.
+template <int CB, int RB, bool BAL, int CH, bool PAYJ>
+__device__ __forceinline__ void round_full(pk2 (&Ih)[CB], pk2 (&Jh)[CB], pk2 cI, pk2 cJ, const BlockPos &q, int s, int n) {
   pk2(&Z)[CB] = PAYJ ? Jh : Ih;
   if (q.publish) {
-    static_for<CB - 1>([&](auto J) { sts64<CECA_IDX(J) * kBkRowBytes>(q.own, Z[CECA_IDX(J)]); });
-    if (q.full_block) sts64<(CB - 1) * kBkRowBytes>(q.own, Z[CB - 1]);
+    static_for<CB - 1>([&](auto J) { sts64<CECA_IDX(J) * RB>(q.own, Z[CECA_IDX(J)]); });
+    if (!BAL || q.full) sts64<(CB - 1) * RB>(q.own, Z[CB - 1]);
     __syncthreads();
   }
   const int first = q.i0 - s;  // source row of offset 0, before the wrap-around
-  if (first >= 0 || first + q.cnt <= 0) {  // the whole block on one side of the wrap-around
-    const uint32_t src = q.col + (uint32_t)((first >= 0 ? first : first + q.n) * kBkRowBytes);
-    constexpr int kChunk = 8;
+  if (first >= 0 || first + q.cnt <= 0) {  // the real rows of the block all on one side of the wrap-around
+    const uint32_t src = q.col + (uint32_t)((first >= 0 ? first : first + n) * RB);
+    constexpr int kChunk = CH;
     static_for<(CB + kChunk - 1) / kChunk>([&](auto C) {
       constexpr int J0 = CECA_IDX(C) * kChunk;
       constexpr int JN = CB - J0 < kChunk ? CB - J0 : kChunk;
       pk2 R[JN];
       static_for<JN>([&](auto J) {
         constexpr int row = J0 + CECA_IDX(J);
-        if constexpr (row < CB - 1) R[CECA_IDX(J)] = lds64<row * kBkRowBytes>(src);
-        else R[CECA_IDX(J)] = q.full_block ? lds64<row * kBkRowBytes>(src) : 0ull;
+        if constexpr (!BAL || row < CB - 1) R[CECA_IDX(J)] = lds64<row * RB>(src);
+        else R[CECA_IDX(J)] = q.full ? lds64<row * RB>(src) : 0ull;   // balanced: row CB-1 of a short block may lie outside the tile
       });
       static_for<JN>([&](auto J) {
         Ih[J0 + CECA_IDX(J)] = axpy2(cI, R[CECA_IDX(J)], Ih[J0 + CECA_IDX(J)]);
@@ -200,8 +218,8 @@ __device__ __forceinline__ void round_full(pk2 (&Ih)[CB], pk2 (&Jh)[CB], pk2 cI,
 #pragma unroll
     for (int j = 0; j < CB; ++j) {
       int row = first + j;
-      if (row < 0) row += q.n;
-      const pk2 r = (j < q.cnt) ? lds64<0>(q.col + (uint32_t)(row * kBkRowBytes)) : 0ull;
+      if (row < 0) row += n;
+      const pk2 r = (j < q.cnt) ? lds64<0>(q.col + (uint32_t)(row * RB)) : 0ull;
       Ih[j] = axpy2(cI, r, Ih[j]);
       Jh[j] = axpy2(cJ, r, Jh[j]);
     }
@@ -210,19 +228,19 @@ __device__ __forceinline__ void round_full(pk2 (&Ih)[CB], pk2 (&Jh)[CB], pk2 cI,
 
 // `sel` (formed on the host): 0 / 1 = every row through shared memory, payload I / J;
 // 2 S + (0 / 1) = the in-register form with shift S, payload I / J.
-template <int CB>
-__device__ __forceinline__ void dispatch_round(int sel, int s, pk2 (&Ih)[CB], pk2 (&Jh)[CB], pk2 cI, pk2 cJ,
+template <int CB, int RB, bool BAL, int CH>
+__device__ __forceinline__ void dispatch_round(int sel, int s, int n, pk2 (&Ih)[CB], pk2 (&Jh)[CB], pk2 cI, pk2 cJ,
                                                const BlockPos &q) {
 #define CECA_BK_CASE(S)                                                              \
   case 2 * S:                                                                        \
-    if constexpr (S < CB) round_partial<CB, S, false>(Ih, Jh, cI, cJ, q);            \
+    if constexpr (S < CB) round_partial<CB, RB, BAL, CH, S, false>(Ih, Jh, cI, cJ, q);        \
     break;                                                                           \
   case 2 * S + 1:                                                                    \
-    if constexpr (S < CB) round_partial<CB, S, true>(Ih, Jh, cI, cJ, q);             \
+    if constexpr (S < CB) round_partial<CB, RB, BAL, CH, S, true>(Ih, Jh, cI, cJ, q);         \
     break;
   switch (sel) {
-    case 0: round_full<CB, false>(Ih, Jh, cI, cJ, q, s); break;
-    case 1: round_full<CB, true>(Ih, Jh, cI, cJ, q, s); break;
+    case 0: round_full<CB, RB, BAL, CH, false>(Ih, Jh, cI, cJ, q, s, n); break;
+    case 1: round_full<CB, RB, BAL, CH, true>(Ih, Jh, cI, cJ, q, s, n); break;
     CECA_BK_CASE(1) CECA_BK_CASE(2) CECA_BK_CASE(3) CECA_BK_CASE(4) CECA_BK_CASE(5) CECA_BK_CASE(6) CECA_BK_CASE(7)
     CECA_BK_CASE(8) CECA_BK_CASE(9) CECA_BK_CASE(10) CECA_BK_CASE(11) CECA_BK_CASE(12) CECA_BK_CASE(13)
     CECA_BK_CASE(14) CECA_BK_CASE(15) CECA_BK_CASE(16) CECA_BK_CASE(17) CECA_BK_CASE(18) CECA_BK_CASE(19)
@@ -232,32 +250,42 @@ __device__ __forceinline__ void dispatch_round(int sel, int s, pk2 (&Ih)[CB], pk
 #undef CECA_BK_CASE
 }
 
-// The number of warps (blocks of agents) per CTA is a launch parameter; MAXT only bounds it and
-// thereby sets the register budget (65536 / MAXT registers per thread).
-template <int CB, int MAXT>
+// CB agents per block, LPB threads (column pairs) per block.  The number of threads per CTA is a
+// launch parameter; MAXT only bounds it and thereby sets the register budget (65536 / MAXT registers
+// per thread).
+template <int CB, int LPB, int MAXT>
 __global__ void __launch_bounds__(MAXT, 1)
 consensus_block_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_y,
                        const __grid_constant__ BlockArgs p) {
+  constexpr int kTileCols = 2 * LPB;
+  constexpr int RB = kTileCols * (int)sizeof(float);
+  constexpr bool kBalanced = LPB >= 16;
+  // received rows in flight per thread: eight, or four where the state leaves fewer than 36 other registers
+  constexpr int kInFlight = 65536 / MAXT - 4 * CB >= 36 ? 8 : 4;
   extern __shared__ __align__(128) unsigned char smem_raw[];
   __shared__ __align__(8) uint64_t bar;
   const int n = p.n;
-  const int lane = threadIdx.x & 31, part = threadIdx.x >> 5;
-  const uint32_t tile_bytes = (uint32_t)n * kBkRowBytes;
-  // [n][64] tiles: landed X, exchange tile of the odd rounds, of the even rounds (the same tile when
-  // there is only one), landed Y (when Y is read)
+  const int lane = threadIdx.x % LPB;       // column pair inside the tile
+  const int part = LPB == 32 ? (int)(threadIdx.x / LPB) : min((int)(threadIdx.x / LPB), p.blocks - 1);
+  // tiles of p.tile_bytes each: 0 = landed X, 1 = exchange tile of the odd rounds, 2 = of the even
+  // rounds (tile 1 again when there is only one), then landed Y (when Y is read).  Tile addresses are
+  // formed where they are used, from the kernel parameters, to keep registers for the state.
   const uint32_t sm_land_x = smem_u32(smem_raw);
-  const uint32_t sm_xch_a = sm_land_x + tile_bytes, sm_xch_b = p.single_xch ? sm_xch_a : sm_xch_a + tile_bytes;
   const uint32_t y_tile = p.single_xch ? 2u : 3u;
-  const uint32_t sm_land_y = sm_land_x + y_tile * tile_bytes;
 
   BlockPos q;
-  q.n = n;
-  q.full_block = part < p.nfull;
-  q.cnt = q.full_block ? CB : CB - 1;
-  q.i0 = q.full_block ? part * CB : p.nfull * CB + (part - p.nfull) * (CB - 1);
+  if (kBalanced) {
+    q.full = part < p.nfull;
+    q.cnt = q.full ? CB : CB - 1;
+    q.i0 = q.full ? part * CB : p.nfull * CB + (part - p.nfull) * (CB - 1);
+  } else {
+    q.i0 = part * CB;
+    q.cnt = min(CB, n - q.i0);
+    q.full = q.cnt == CB;
+  }
   const uint32_t col_off = 2u * lane * (uint32_t)sizeof(float);
-  const uint32_t own_off = (uint32_t)q.i0 * kBkRowBytes + col_off;
-  const uint32_t prev_off = (uint32_t)(part == 0 ? n : q.i0) * kBkRowBytes + col_off;
+  const uint32_t own_off = (uint32_t)q.i0 * RB + col_off;
+  const uint32_t prev_off = (uint32_t)(part == 0 ? n : q.i0) * RB + col_off;
 
   if (threadIdx.x == 0) {
     mbar_init(&bar, 1);
@@ -267,14 +295,16 @@ consensus_block_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
 
   auto issue_load = [&](int32_t tile) {
     mbar_expect_tx(&bar, p.tx_bytes);
-    tma_load_2d(smem_raw, &map_x, tile * kBkTileCols, 0, &bar);
-    if (p.has_y_in) tma_load_2d(smem_raw + (size_t)y_tile * tile_bytes, &map_y, tile * kBkTileCols, 0, &bar);
+    for (int b = 0; b < p.boxes; ++b) {   // rows past n are outside the tensor map: they read as zero
+      const int row0 = b * p.box_rows;
+      tma_load_2d(smem_raw + (size_t)row0 * RB, &map_x, tile * kTileCols, row0, &bar);
+      if (p.has_y_in)
+        tma_load_2d(smem_raw + (size_t)y_tile * p.tile_bytes + (size_t)row0 * RB, &map_y, tile * kTileCols, row0, &bar);
+    }
   };
   if (threadIdx.x == 0 && (int32_t)blockIdx.x < p.tiles) issue_load((int32_t)blockIdx.x);
 
   const bool prefetch_in_loop = p.rounds > 2;
-  float *const dst_x = p.Xo + (int64_t)q.i0 * p.ld + 2 * lane;
-  float *const dst_y = p.Yo + (int64_t)q.i0 * p.ld + 2 * lane;
 
   uint32_t phase = 0;
   for (int32_t tile = blockIdx.x; tile < p.tiles; tile += gridDim.x) {
@@ -291,16 +321,28 @@ consensus_block_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
 
     pk2 Ih[CB], Jh[CB];
     {
-      const uint32_t own = sm_land_x + own_off;
-      static_for<CB - 1>([&](auto J) { Ih[CECA_IDX(J)] = lds64<CECA_IDX(J) * kBkRowBytes>(own); });
-      Ih[CB - 1] = q.full_block ? lds64<(CB - 1) * kBkRowBytes>(own) : 0ull;
-      if (p.has_y_in) {
-        const uint32_t owny = sm_land_y + own_off;
-        static_for<CB - 1>([&](auto J) { Jh[CECA_IDX(J)] = lds64<CECA_IDX(J) * kBkRowBytes>(owny); });
-        Jh[CB - 1] = q.full_block ? lds64<(CB - 1) * kBkRowBytes>(owny) : 0ull;
+      // balanced cut: only row CB-1 may be missing; uniform cut: any number of rows of the last block
+      const uint32_t own = sm_land_x + own_off, owny = own + y_tile * p.tile_bytes;
+      if (!kBalanced && q.full) {
+        static_for<CB>([&](auto J) { Ih[CECA_IDX(J)] = lds64<CECA_IDX(J) * RB>(own); });
       } else {
+        static_for<CB>([&](auto J) {
+          constexpr int j = CECA_IDX(J);
+          if constexpr (kBalanced && j < CB - 1) Ih[j] = lds64<j * RB>(own);
+          else Ih[j] = (q.full || j < q.cnt) ? lds64<j * RB>(own) : 0ull;
+        });
+      }
+      if (!p.has_y_in) {
 #pragma unroll
         for (int j = 0; j < CB; ++j) Jh[j] = 0ull;
+      } else if (!kBalanced && q.full) {
+        static_for<CB>([&](auto J) { Jh[CECA_IDX(J)] = lds64<CECA_IDX(J) * RB>(owny); });
+      } else {
+        static_for<CB>([&](auto J) {
+          constexpr int j = CECA_IDX(J);
+          if constexpr (kBalanced && j < CB - 1) Jh[j] = lds64<j * RB>(owny);
+          else Jh[j] = (q.full || j < q.cnt) ? lds64<j * RB>(owny) : 0ull;
+        });
       }
     }
     const int32_t next_tile = tile + (int32_t)gridDim.x;
@@ -326,27 +368,41 @@ consensus_block_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
       }
       // The first round finds every row's payload in the landed tile and publishes nothing.
       q.publish = rnd > 0;
-      const uint32_t buf = rnd == 0 ? ((mode & kBkPayloadJ) ? sm_land_y : sm_land_x) : ((rnd & 1) ? sm_xch_a : sm_xch_b);
+      const uint32_t buf_tile = rnd == 0 ? ((mode & kBkPayloadJ) ? y_tile : 0u) : ((rnd & 1) || p.single_xch ? 1u : 2u);
+      const uint32_t buf = sm_land_x + buf_tile * p.tile_bytes;
       q.own = buf + own_off;
       q.prev = buf + prev_off;
       q.col = buf + col_off;
-      dispatch_round<CB>(rd.sel, rd.hop, Ih, Jh, pk_make(rd.cI, rd.cI), pk_make(rd.cJ, rd.cJ), q);
+      dispatch_round<CB, RB, kBalanced, kInFlight>(rd.sel, rd.hop, p.n, Ih, Jh, pk_make(rd.cI, rd.cI), pk_make(rd.cJ, rd.cJ), q);
       // with a single exchange tile the next round's publish must wait for this round's reads
       if (p.single_xch && rnd >= 1 && rnd + 1 < p.rounds) __syncthreads();
     }
 
-    const int32_t col = tile * kBkTileCols + 2 * lane;
-    if (col + 1 < p.d) {
+    const int32_t col = tile * kTileCols + 2 * lane;
+    // surplus threads (only where a block is narrower than a warp) shadow the last block and write nothing
+    if (LPB < 32 && (int)(threadIdx.x / LPB) >= p.blocks) {
+    } else if (col + 1 < p.d) {
       const pk2 oI = pk_make(p.outI, p.outI), oJ = pk_make(p.outJ, p.outJ);
-      float *dst = dst_x + col - 2 * lane;
+      float *dst = p.Xo + (int64_t)q.i0 * p.ld + col;
+      float *dsty = p.Yo + (int64_t)q.i0 * p.ld + col;
+      if (!kBalanced && q.full) {
 #pragma unroll
-      for (int j = 0; j < CB - 1; ++j) __stcs(reinterpret_cast<pk2 *>(dst + j * p.ld), mul2(oI, Ih[j]));
-      if (q.full_block) __stcs(reinterpret_cast<pk2 *>(dst + (CB - 1) * p.ld), mul2(oI, Ih[CB - 1]));
-      if (p.has_y_out) {
-        float *dsty = dst_y + col - 2 * lane;
+        for (int j = 0; j < CB; ++j) __stcs(reinterpret_cast<pk2 *>(dst + j * p.ld), mul2(oI, Ih[j]));
+        if (p.has_y_out) {
 #pragma unroll
-        for (int j = 0; j < CB - 1; ++j) __stcs(reinterpret_cast<pk2 *>(dsty + j * p.ld), mul2(oJ, Jh[j]));
-        if (q.full_block) __stcs(reinterpret_cast<pk2 *>(dsty + (CB - 1) * p.ld), mul2(oJ, Jh[CB - 1]));
+          for (int j = 0; j < CB; ++j) __stcs(reinterpret_cast<pk2 *>(dsty + j * p.ld), mul2(oJ, Jh[j]));
+        }
+      } else {
+        static_for<CB>([&](auto J) {
+          constexpr int j = CECA_IDX(J);
+          if ((kBalanced && j < CB - 1) || q.full || j < q.cnt) __stcs(reinterpret_cast<pk2 *>(dst + j * p.ld), mul2(oI, Ih[j]));
+        });
+        if (p.has_y_out) {
+          static_for<CB>([&](auto J) {
+            constexpr int j = CECA_IDX(J);
+            if ((kBalanced && j < CB - 1) || q.full || j < q.cnt) __stcs(reinterpret_cast<pk2 *>(dsty + j * p.ld), mul2(oJ, Jh[j]));
+          });
+        }
       }
     } else if (col < p.d) {   // d odd: the last column has no partner
 #pragma unroll
@@ -366,16 +422,78 @@ consensus_block_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
 
 // ---- host side ----------------------------------------------------------------------------------
 
-constexpr int kBkMaxRows = 256;
 constexpr size_t kBkSmemLimit = 227 * 1024 - 1024;   // opt-in maximum per CTA minus the static part
+
+// Geometry by n: threads per block of agents (tile = 2 * LPB columns), number of blocks, agents per block.
+//   LPB = 32 (n <= 256): blocks are warps; as few and as large as the register file allows (25 agents
+//     take 100 state registers), because a round whose shift reaches the block size exchanges every
+//     row through shared memory and there are about log2(blocks) such rounds; 1, 2 or a multiple of 4
+//     warps, so that the warps of a CTA, which move in lockstep from barrier to barrier, load the four
+//     schedulers of an SM evenly (5, 6, 7 or 9 warps measured 15-40 % slower than 4 or 8).
+//   LPB = 16 (n <= 512), LPB = 8 (n <= 1152): narrower tiles, so that all n rows of a tile (three
+//     tiles' worth: landed, two exchange tiles) still fit in shared memory, in at most 512 threads.
+//     LPB = 8 takes an odd CB from a short list (see the bank argument at the top).
+struct BlockGeom {
+  int lpb, cb, blocks, threads;
+  int nfull;   // see BlockArgs
+  int cmin;    // size of the smallest block that a partial round's source rows may lie in
+};
+constexpr int kBkMaxRows = 1152;
+static bool block_geometry(int n, int warps_override, BlockGeom *g) {
+  if (n < 2 || n > kBkMaxRows) return false;
+  if (n <= 512) {
+    int blocks;
+    if (n <= 256) {
+      g->lpb = 32;
+      blocks = n <= 25 ? 1 : n <= 50 ? 2 : n <= 100 ? 4 : n <= 200 ? 8 : 12;
+      if (warps_override > 0) blocks = warps_override;
+    } else {
+      g->lpb = 16;
+      blocks = n <= 336 ? 16 : n <= 504 ? 24 : 32;
+    }
+    if (blocks > n) blocks = n;
+    g->blocks = blocks;
+    g->cb = (n + blocks - 1) / blocks;
+    g->nfull = n - blocks * (g->cb - 1);          // 1 .. blocks
+    g->cmin = g->nfull == blocks ? g->cb : g->cb - 1;
+  } else {
+    g->lpb = 8;
+    static const int kSizes[] = {9, 13, 17, 21, 25};
+    g->cb = 0;
+    for (int cb : kSizes)
+      if ((n + cb - 1) / cb <= 512 / g->lpb) { g->cb = cb; break; }
+    if (!g->cb) return false;
+    g->blocks = (n + g->cb - 1) / g->cb;
+    g->nfull = n / g->cb;
+    g->cmin = g->cb;   // the sources of a partial round lie in full blocks, or are all published (last block)
+  }
+  if (g->cb > 25) return false;
+  g->threads = (g->blocks * g->lpb + 31) / 32 * 32;
+  return true;
+}
+
+struct BlockTile {
+  int boxes, box_rows;
+  size_t tile_bytes;
+};
+static BlockTile block_tile(int n, const BlockGeom &g) {
+  BlockTile t;
+  const int row_bytes = 2 * g.lpb * (int)sizeof(float);
+  t.boxes = (n + kBkMaxBoxRows - 1) / kBkMaxBoxRows;
+  t.box_rows = (n + t.boxes - 1) / t.boxes;
+  if (t.boxes > 1) t.box_rows = (t.box_rows + 1) / 2 * 2;   // every box starts on a 128-byte boundary of shared memory
+  int rows = t.boxes * t.box_rows;
+  if (g.lpb == 8 && g.blocks * g.cb > rows) rows = g.blocks * g.cb;   // phantom rows of the last block stay inside the tile
+  t.tile_bytes = ((size_t)rows * row_bytes + 127) / 128 * 128;
+  return t;
+}
 
 // y_in: the first round reads Y, which takes one more shared-memory tile (at least two are needed without it).
 bool consensus_block_supports(int32_t n, ceca_variant_t variant, int32_t rounds, bool y_in) {
-  return variant == CECA_2P && n >= 2 && n <= kBkMaxRows && rounds >= 1 && rounds <= kBkMaxRounds &&
-         (size_t)(y_in ? 3 : 2) * n * kBkTileCols * sizeof(float) <= kBkSmemLimit;
+  BlockGeom g;
+  if (variant != CECA_2P || rounds < 1 || rounds > kBkMaxRounds || !block_geometry(n, 0, &g)) return false;
+  return (size_t)(y_in ? 3 : 2) * block_tile(n, g).tile_bytes <= kBkSmemLimit;
 }
-
-constexpr int kBkMaxWarps = 12;   // 12 blocks of 22 agents cover n = 256
 
 // Register budgets by block size (the state takes 4 * CB registers): a roomy one, and a lean one that
 // still compiles without spilling to speak of.  65536 / kMaxThreads registers per thread.
@@ -384,15 +502,15 @@ template <int CB> struct BlockRegs {
   static constexpr int kLean = CB >= 15 ? 512 : CB >= 11 ? 768 : 1024;
 };
 
-template <int CB, int MAXT>
-static cudaError_t launch_block_regs(const CUtensorMap &mx, const CUtensorMap &my, const BlockArgs &a, int warps,
+template <int CB, int LPB, int MAXT>
+static cudaError_t launch_block_regs(const CUtensorMap &mx, const CUtensorMap &my, const BlockArgs &a, int threads,
                                      size_t smem, int *per_sm_out, bool launch, cudaStream_t stream) {
   static std::atomic<uint64_t> attr_done{0};
-  cudaError_t e = set_max_shared_once(reinterpret_cast<const void *>(consensus_block_kernel<CB, MAXT>), kBkSmemLimit,
-                                      &attr_done);
+  cudaError_t e = set_max_shared_once(reinterpret_cast<const void *>(consensus_block_kernel<CB, LPB, MAXT>),
+                                      kBkSmemLimit, &attr_done);
   if (e != cudaSuccess) return e;
   int per_sm = 0;
-  e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, consensus_block_kernel<CB, MAXT>, 32 * warps, smem);
+  e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, consensus_block_kernel<CB, LPB, MAXT>, threads, smem);
   if (e != cudaSuccess) return e;
   *per_sm_out = per_sm;
   if (!launch) return cudaSuccess;
@@ -402,23 +520,19 @@ static cudaError_t launch_block_regs(const CUtensorMap &mx, const CUtensorMap &m
   // persistent CTAs: as many as fit on the device at once, not more than there are tiles
   const int64_t resident = (int64_t)sms * per_sm;
   const int grid = (int)(a.tiles < resident ? a.tiles : resident);
-  consensus_block_kernel<CB, MAXT><<<grid, 32 * warps, smem, stream>>>(mx, my, a);
+  consensus_block_kernel<CB, LPB, MAXT><<<grid, threads, smem, stream>>>(mx, my, a);
   return cudaGetLastError();
 }
 
-template <int CB>
-static cudaError_t launch_block(const CUtensorMap &mx, const CUtensorMap &my, BlockArgs &a, int warps,
+template <int CB, int LPB>
+static cudaError_t launch_block(const CUtensorMap &mx, const CUtensorMap &my, BlockArgs &a, int threads, int cmin,
                                 cudaStream_t stream) {
-  const int n = a.n;
-  a.nfull = n - warps * (CB - 1);
-  const int cmin = a.nfull == warps ? CB : CB - 1;
   for (int t = 0; t < a.rounds; ++t) {
     BlockRound &r = a.rd[t];
     const int pay = (r.mode & kBkPayloadJ) ? 1 : 0;
     r.sel = r.hop < cmin ? 2 * r.hop + pay : pay;   // in-register form while the shift is smaller than every block
   }
-  const size_t tile_bytes = (size_t)n * kBkTileCols * sizeof(float);
-  if (32 * warps > BlockRegs<CB>::kRoomy) return cudaErrorInvalidConfiguration;
+  const size_t tile_bytes = a.tile_bytes;
   // Four candidates: two or one exchange tile, roomy or lean register budget.  The default is two tiles
   // and the roomy budget; an alternative is taken only when it lets more CTAs share an SM.
   constexpr int kRoomy = BlockRegs<CB>::kRoomy, kLean = BlockRegs<CB>::kLean;
@@ -427,10 +541,12 @@ static cudaError_t launch_block(const CUtensorMap &mx, const CUtensorMap &my, Bl
     const size_t smem = ((a.has_y_in ? 2 : 1) + (single ? 1 : 2)) * tile_bytes;
     if (smem > kBkSmemLimit) continue;
     int roomy = 0, lean = 0;
-    cudaError_t e = launch_block_regs<CB, kRoomy>(mx, my, a, warps, smem, &roomy, false, stream);
-    if (e != cudaSuccess) return e;
-    if (kLean != kRoomy) {
-      e = launch_block_regs<CB, kLean>(mx, my, a, warps, smem, &lean, false, stream);
+    if (threads <= kRoomy) {
+      cudaError_t e = launch_block_regs<CB, LPB, kRoomy>(mx, my, a, threads, smem, &roomy, false, stream);
+      if (e != cudaSuccess) return e;
+    }
+    if (kLean != kRoomy && threads <= kLean) {
+      cudaError_t e = launch_block_regs<CB, LPB, kLean>(mx, my, a, threads, smem, &lean, false, stream);
       if (e != cudaSuccess) return e;
     }
     if (roomy > best) { best = roomy; best_single = single; best_lean = 0; }
@@ -440,24 +556,14 @@ static cudaError_t launch_block(const CUtensorMap &mx, const CUtensorMap &my, Bl
   a.single_xch = best_single;
   const size_t smem = ((a.has_y_in ? 2 : 1) + (best_single ? 1 : 2)) * tile_bytes;
   int per_sm = 0;
-  if (best_lean) return launch_block_regs<CB, kLean>(mx, my, a, warps, smem, &per_sm, true, stream);
-  return launch_block_regs<CB, kRoomy>(mx, my, a, warps, smem, &per_sm, true, stream);
-}
-
-// Blocks (= warps) per CTA for n agents.  As few, i.e. as large, as the register file allows (25
-// agents take 100 state registers), because a round whose shift reaches the block size exchanges
-// every row through shared memory and there are about log2(blocks) such rounds; and 1, 2 or a
-// multiple of 4, so that the warps of a CTA, which move in lockstep from barrier to barrier, load
-// the four schedulers of an SM evenly (5, 6, 7 or 9 warps measured 15-40 % slower than 4 or 8).
-// `warps_override` > 0 forces a value (used to measure the alternatives).
-static int block_warps(int n, int warps_override) {
-  if (warps_override > 0) return warps_override;
-  return n <= 25 ? 1 : n <= 50 ? 2 : n <= 100 ? 4 : n <= 200 ? 8 : 12;
+  if (best_lean) return launch_block_regs<CB, LPB, kLean>(mx, my, a, threads, smem, &per_sm, true, stream);
+  return launch_block_regs<CB, LPB, kRoomy>(mx, my, a, threads, smem, &per_sm, true, stream);
 }
 
 // Arguments are assumed validated by the caller (shapes, aliasing, 16-byte alignment of X / Y and
 // ld % 4 == 0, d and ld within 32 bits, Y present when the first round reads it, status word).
-// The caller has checked consensus_block_supports.
+// The caller has checked consensus_block_supports.  `warps_override` > 0 forces the number of
+// blocks for n <= 256 (used to measure the alternatives).
 ceca_status_t consensus_block(const float *X, const float *Y, float *Xo, float *Yo, int32_t n, int64_t d,
                               int64_t ld, int64_t k0, int32_t rounds, int32_t *status, int32_t wait_polls,
                               uint32_t tx_extra, int warps_override, cudaStream_t stream) {
@@ -465,7 +571,6 @@ ceca_status_t consensus_block(const float *X, const float *Y, float *Xo, float *
   std::memset(&a, 0, sizeof(a));
   a.Xo = Xo; a.Yo = Yo; a.ld = ld; a.d = (int32_t)d; a.n = n; a.rounds = rounds;
   a.has_y_out = Yo ? 1 : 0;
-  a.tiles = (int32_t)((d + kBkTileCols - 1) / kBkTileCols);
   a.status = status;
   a.wait_polls = wait_polls > 0 ? wait_polls : (int32_t)kBkWaitPolls;
 
@@ -493,25 +598,48 @@ ceca_status_t consensus_block(const float *X, const float *Y, float *Xo, float *
   }
   a.outI = (float)alpha; a.outJ = (float)beta;
   a.has_y_in = (Y != nullptr && first_needs_y) ? 1 : 0;
-  a.tx_bytes = (uint32_t)n * kBkTileCols * sizeof(float) * (a.has_y_in ? 2u : 1u) + tx_extra;
   if (!consensus_block_supports(n, CECA_2P, rounds, a.has_y_in != 0)) return CECA_ERR_UNSUPPORTED;
 
-  CUtensorMap mx, my;
-  if (!tensor_map_2d(&mx, X, n, d, ld, kBkTileCols, n)) return CECA_ERR_CUDA;
-  if (!tensor_map_2d(&my, a.has_y_in ? Y : X, n, d, ld, kBkTileCols, n)) return CECA_ERR_CUDA;
+  BlockGeom g;
+  if (!block_geometry(n, warps_override, &g)) return CECA_ERR_UNSUPPORTED;
+  const BlockTile t = block_tile(n, g);
+  const int tile_cols = 2 * g.lpb;
+  a.blocks = g.blocks; a.nfull = g.nfull; a.boxes = t.boxes; a.box_rows = t.box_rows; a.tile_bytes = (uint32_t)t.tile_bytes;
+  a.tiles = (int32_t)((d + tile_cols - 1) / tile_cols);
+  // a box counts in full towards the barrier, rows and columns outside the matrix included
+  a.tx_bytes = (uint32_t)t.boxes * t.box_rows * tile_cols * sizeof(float) * (a.has_y_in ? 2u : 1u) + tx_extra;
 
-  const int warps = block_warps(n, warps_override);
-  if (warps < 1 || warps > kBkMaxWarps) return CECA_ERR_UNSUPPORTED;
+  CUtensorMap mx, my;
+  if (!tensor_map_2d(&mx, X, n, d, ld, tile_cols, t.box_rows)) return CECA_ERR_CUDA;
+  if (!tensor_map_2d(&my, a.has_y_in ? Y : X, n, d, ld, tile_cols, t.box_rows)) return CECA_ERR_CUDA;
+
   cudaError_t e = cudaErrorInvalidConfiguration;
-  switch ((n + warps - 1) / warps) {   // agents per block
-#define CECA_BK_LAUNCH(CB) case CB: e = launch_block<CB>(mx, my, a, warps, stream); break;
-    CECA_BK_LAUNCH(1) CECA_BK_LAUNCH(2) CECA_BK_LAUNCH(3) CECA_BK_LAUNCH(4) CECA_BK_LAUNCH(5) CECA_BK_LAUNCH(6)
-    CECA_BK_LAUNCH(7) CECA_BK_LAUNCH(8) CECA_BK_LAUNCH(9) CECA_BK_LAUNCH(10) CECA_BK_LAUNCH(11) CECA_BK_LAUNCH(12)
-    CECA_BK_LAUNCH(13) CECA_BK_LAUNCH(14) CECA_BK_LAUNCH(15) CECA_BK_LAUNCH(16) CECA_BK_LAUNCH(17) CECA_BK_LAUNCH(18)
-    CECA_BK_LAUNCH(19) CECA_BK_LAUNCH(20) CECA_BK_LAUNCH(21) CECA_BK_LAUNCH(22) CECA_BK_LAUNCH(23) CECA_BK_LAUNCH(24)
-    CECA_BK_LAUNCH(25)
+  if (g.lpb == 32) {
+    switch (g.cb) {
+#define CECA_BK_LAUNCH(CB) case CB: e = launch_block<CB, 32>(mx, my, a, g.threads, g.cmin, stream); break;
+      CECA_BK_LAUNCH(1) CECA_BK_LAUNCH(2) CECA_BK_LAUNCH(3) CECA_BK_LAUNCH(4) CECA_BK_LAUNCH(5) CECA_BK_LAUNCH(6)
+      CECA_BK_LAUNCH(7) CECA_BK_LAUNCH(8) CECA_BK_LAUNCH(9) CECA_BK_LAUNCH(10) CECA_BK_LAUNCH(11) CECA_BK_LAUNCH(12)
+      CECA_BK_LAUNCH(13) CECA_BK_LAUNCH(14) CECA_BK_LAUNCH(15) CECA_BK_LAUNCH(16) CECA_BK_LAUNCH(17) CECA_BK_LAUNCH(18)
+      CECA_BK_LAUNCH(19) CECA_BK_LAUNCH(20) CECA_BK_LAUNCH(21) CECA_BK_LAUNCH(22) CECA_BK_LAUNCH(23) CECA_BK_LAUNCH(24)
+      CECA_BK_LAUNCH(25)
 #undef CECA_BK_LAUNCH
-    default: break;
+      default: break;
+    }
+  } else if (g.lpb == 16) {
+#define CECA_BK_LAUNCH(CB) case CB: e = launch_block<CB, 16>(mx, my, a, g.threads, g.cmin, stream); break;
+    switch (g.cb) {   // n = 257 .. 512 in 16, 24 or 32 blocks: 15 to 21 agents per block
+      CECA_BK_LAUNCH(15) CECA_BK_LAUNCH(16) CECA_BK_LAUNCH(17) CECA_BK_LAUNCH(18) CECA_BK_LAUNCH(19) CECA_BK_LAUNCH(20)
+      CECA_BK_LAUNCH(21)
+      default: break;
+    }
+#undef CECA_BK_LAUNCH
+  } else {
+#define CECA_BK_LAUNCH(CB) case CB: e = launch_block<CB, 8>(mx, my, a, g.threads, g.cmin, stream); break;
+    switch (g.cb) {
+      CECA_BK_LAUNCH(9) CECA_BK_LAUNCH(13) CECA_BK_LAUNCH(17) CECA_BK_LAUNCH(21) CECA_BK_LAUNCH(25)
+      default: break;
+    }
+#undef CECA_BK_LAUNCH
   }
   if (e == cudaErrorInvalidConfiguration) return CECA_ERR_UNSUPPORTED;
   return e == cudaSuccess ? CECA_OK : CECA_ERR_CUDA;

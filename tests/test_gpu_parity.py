@@ -256,17 +256,20 @@ def test_mean_lemma_and_resume_on_gpu(n, variant):
 # consensus rounds: one launch per round, and the fused TMA kernel
 # --------------------------------------------------------------------------------------------
 
+BLOCK_MAX_N = 1152   # largest n the register-block kernel takes (16-column tiles of all rows on one SM)
+
+
 def _fused_ws():
     return torch.zeros(64, dtype=torch.int32, device=DEV)
 
 
 def _fused_kernels(n, variant=ceca.CECA_2P):
     """The fused kernels that take n agents and this variant: shared-memory exchange (n <= 2048),
-    tensor-memory exchange (n <= 128), register blocks (CECA-2P, n <= 256)."""
+    tensor-memory exchange (n <= 128), register blocks (CECA-2P, n <= 1152)."""
     kernels = [ceca.FUSED_SMEM]
     if n <= 128:
         kernels.append(ceca.FUSED_TMEM)
-    if n <= 256 and variant == ceca.CECA_2P:
+    if n <= BLOCK_MAX_N and variant == ceca.CECA_2P:
         kernels.append(ceca.FUSED_BLOCK)
     return kernels
 
@@ -310,19 +313,25 @@ def test_consensus_matches_oracle_and_reaches_the_mean(fused, n, d):
             assert torch.equal(X, Xo) and torch.equal(Y, Yo)
 
 
-@pytest.mark.parametrize("n", [257, 300, 514, 1026, 1300, 2047, 2048])
+@pytest.mark.parametrize("fused", [ceca.FUSED_AUTO, ceca.FUSED_SMEM, ceca.FUSED_BLOCK])
+@pytest.mark.parametrize("n", [257, 258, 300, 511, 512, 513, 514, 1026, 1087, 1088, 1089, 1152, 1153, 1300, 2047, 2048])
 @pytest.mark.parametrize("d", [8, 1000, 4100])
-def test_fused_consensus_above_256_agents(n, d):
-    """Narrow (8-column) tiles made of several TMA boxes: tau rounds, extra rounds, unaligned starts."""
+def test_fused_consensus_above_256_agents(fused, n, d):
+    """Tiles taller than one TMA box (32-, 16- or 8-column tiles made of several boxes): tau rounds, extra rounds,
+    unaligned starts; every fused kernel that takes this n, and the one the library picks by itself."""
     x = synth.consensus_inputs(n, d, seed=n + d)
     y0 = synth.consensus_inputs(n, d, seed=n + d + 1, offset_rows=False)
     tau = _tau(n)
     for variant in _variants(n):
-        for k0, rounds in [(0, tau), (3, tau + 2), (tau, 1)]:
+        if fused == ceca.FUSED_BLOCK and fused not in _fused_kernels(n, variant):
+            with pytest.raises(ceca.CecaError):   # outside that kernel's range: refused, nothing launched
+                ceca.ceca_consensus_rounds(x.to(DEV), None, variant, 0, 1, fused, workspace=_fused_ws(), want_y=False)
+            continue
+        for k0, rounds in [(0, tau), (3, tau + 2), (tau, 1), (tau - 1, 2)]:
             X, Y = x.to(DEV), y0.to(DEV)
             Xo, Yo = torch.full_like(X, float("nan")), torch.full_like(Y, float("nan"))
             ws = _fused_ws()
-            ceca.ceca_consensus_rounds(X, Y, variant, k0, rounds, 1, X_out=Xo, Y_out=Yo, workspace=ws)
+            ceca.ceca_consensus_rounds(X, Y, variant, k0, rounds, fused, X_out=Xo, Y_out=Yo, workspace=ws)
             assert ceca.ceca_read_status(ws) == 0
             want_x, want_y = oracle.consensus(_np(x), _np(y0), variant, k0, rounds)
             tol = STEP_TOL * rounds * _scale(0, (x, 1), (y0, 1))
@@ -331,7 +340,7 @@ def test_fused_consensus_above_256_agents(n, d):
             if k0 == 0:
                 xd = Xo.double()
                 assert float((xd - x.double().mean(0).to(DEV)).norm() / xd.norm()) <= 1e-5
-            ceca.ceca_consensus_rounds(X, Y, variant, k0, rounds, 1, workspace=ws)   # in place: same bits
+            ceca.ceca_consensus_rounds(X, Y, variant, k0, rounds, fused, workspace=ws)   # in place: same bits
             assert torch.equal(X, Xo) and torch.equal(Y, Yo)
 
 
