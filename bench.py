@@ -45,6 +45,11 @@ WORKLOADS = {
     # smaller cases of the same kernels, for profiler captures and quick looks
     "resnet18_step": dict(kind="step", n=24, d=11_689_512, variant=1, gamma=0.1),
     "step_small": dict(kind="step", n=100, d=2_097_152, variant=2, gamma=0.1),
+    # rows a multiple of 4 floats apart, but X, Y and G all start one float past a 16-byte boundary (views that
+    # skip the first element of their buffers): a scalar head of 3 columns, then the 128-bit body
+    "step_offset_base": dict(kind="step", n=100, d=4_194_300, variant=2, gamma=0.1, base_offset=1),
+    # nothing to align: ld = d = 4,194,303, every column runs the scalar form
+    "step_odd_ld": dict(kind="step", n=100, d=4_194_303, variant=2, gamma=0.1, ld=4_194_303),
     # n a power of two: the X-only update (12 B per agent-parameter; CECA-2P = one-peer exponential graph)
     "pow2_xonly_step": dict(kind="step", n=128, d=8_388_608, variant=2, gamma=0.1, x_only=True),
     # fused = 1 picks the kernel by n and variant (register blocks for CECA-2P up to n = 1152, shared-memory exchange otherwise)
@@ -61,6 +66,9 @@ WORKLOADS = {
     "consensus_fused_1026_smem": dict(kind="consensus", n=1026, d=1 << 18, variant=2, fused=2),
     "consensus_rounds_1026": dict(kind="consensus", n=1026, d=1 << 18, variant=2, fused=0),
     "logreg_grad": dict(kind="logreg", n=63, m=2000, d=4096, variant=2, gamma=0.01),
+    # wider models at the same 2 GB of samples: clusters of 2 (d = 8192) and 8 (d = 32768) CTAs, 4096 columns each
+    "logreg_grad_d8192": dict(kind="logreg", n=32, m=2000, d=8192, variant=2, gamma=0.01),
+    "logreg_grad_d32768": dict(kind="logreg", n=8, m=2000, d=32768, variant=2, gamma=0.01),
     # whole iterations (gradient kernel + fused step), one CECA cycle captured in a CUDA graph and replayed
     "logreg_train": dict(kind="train", n=63, m=2000, d=4096, variant=2, gamma=0.01, loss="logistic"),
     # the same with a global average (tau + 1 fused consensus rounds) after every second cycle, all inside the graph
@@ -250,8 +258,14 @@ def bench_step(args, wl, device, dist):
     import synthetic_inputs as synth
 
     n, d, variant, gamma = wl["n"], wl["d"], wl["variant"], wl["gamma"]
-    ld = synth.padded_ld(d)  # rows 128-byte aligned: a warp's 512-byte access then covers exactly four lines
-    X, Y, G = synth.step_inputs(n, d, seed=0, x_std=0.01, g_std=0.01, device=device, ld=ld)
+    ld = wl.get("ld") or synth.padded_ld(d)  # rows 128-byte aligned: a warp's 512-byte access then covers exactly four lines
+    off = int(wl.get("base_offset", 0))
+    if off:
+        ld = synth.padded_ld(d + off)
+        X, Y, G = (torch.as_strided(t, (n, d), (ld, 1), storage_offset=off) for t in
+                   synth.step_inputs(n, d + off, seed=0, x_std=0.01, g_std=0.01, device=device, ld=ld))
+    else:
+        X, Y, G = synth.step_inputs(n, d, seed=0, x_std=0.01, g_std=0.01, device=device, ld=ld)
     storage = wl.get("storage", "f32")
     if storage != "f32":   # the same draws, stored narrow (row by row: no second full-size temporary)
         def narrow(t):
@@ -304,7 +318,7 @@ def bench_step(args, wl, device, dist):
                 if not (drop and (k_first + s) % tau == tau - 1)
                 and (x_only or ceca.ceca_schedule(n, variant, k_first + s, peers=False)[0].b_num != 0
                      or ceca.ceca_schedule(n, variant, k_first + s, peers=False)[0].payload == 1)]
-    launches = args.steps * (1 if d % 4 == 0 else 2)
+    launches = args.steps * ((1 if d % 4 == 0 else 2) + (1 if off else 0))
     roof = None
     if dominant:
         avg_ms = sum(dominant) / len(dominant)
@@ -459,7 +473,7 @@ def bench_logreg(args, wl, device, dist):
     roof = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
             "traffic": ncu_traffic(args.workload),
             "kernel": "logreg_fused_kernel + logreg_reduce_kernel", "peak_source": "of " + which, "avg_launch_ms": grad_ms}
-    return total_ms, 3 * args.steps, roof, clocks, {"m": m, "l2": "A is 2.06 GB, larger than L2"}
+    return total_ms, 3 * args.steps, roof, clocks, {"m": m, "l2": "A is %.2f GB, larger than L2" % (4e-9 * n * m * d)}
 
 
 def bench_train(args, wl, device, dist):

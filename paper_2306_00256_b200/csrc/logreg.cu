@@ -6,7 +6,7 @@
 // with z = X if delta_r = 1 else Y.  Both are "coefficient per sample times the sample", so they
 // share the kernels below; only the coefficient differs.
 //
-// Main path (d a multiple of 4, d <= 8192, 16-byte aligned rows): A is read exactly once.  A CTA
+// Main path (d a multiple of 4, d <= 65536, 16-byte aligned rows): A is read exactly once.  A CTA
 // takes one agent and a block of its samples; each thread keeps its slice of z_i and of the
 // running gradient in registers, loads its slice of four sample rows, the CTA reduces the four
 // inner products (warp shuffles, then a fixed-order sum over the warps through shared memory),
@@ -14,9 +14,15 @@
 // gradient slice.  Per-CTA partial gradients go to the workspace and a second kernel adds them in
 // a fixed order, so the result does not change from run to run.  Not a dense contraction worth
 // tensor cores: two matrix-vector products per agent, bound by reading A from HBM.
+// A CTA's registers hold up to 8192 columns.  Wider models run the same kernel as a thread-block
+// cluster of up to eight CTAs, one column chunk each: every CTA writes its share of the inner
+// products into the shared memory of all CTAs of the cluster (distributed shared memory), one
+// cluster barrier makes them visible, and every CTA adds the shares in rank order, so all of them
+// get the same bits.
 //
-// Fallback (any d, any alignment): coefficients first (one warp per sample), then a column-wise
-// accumulation; A is read twice.
+// Fallback (any other d, any alignment): coefficients first (one warp per sample), then a
+// column-wise accumulation; A is read twice.
+#include <cooperative_groups.h>
 #include <cuda_runtime.h>
 
 #include <cstdint>
@@ -29,13 +35,37 @@ namespace ceca {
 
 constexpr int kLrThreads = 256;
 constexpr int kLrWarps = kLrThreads / 32;
-constexpr int kLrSamples = 4;        // sample rows in flight per thread
-constexpr int kLrMaxVpt = 8;         // float4 column groups per thread -> d <= 256*4*8 = 8192
+constexpr int kLrMaxVpt = 8;         // float4 column groups per thread -> 256*4*8 = 8192 columns per CTA
+constexpr int kLrMaxCluster = 8;     // CTAs (column chunks) per cluster: the portable maximum
+constexpr int kLrChunkCols = kLrThreads * 4 * kLrMaxVpt;
+constexpr int kLrHalfChunkCols = kLrChunkCols / 2;   // four float4 per thread: two CTAs per SM, four rows in flight
 constexpr int kLrTargetCtas = 148 * 12;
 
-static inline int32_t logreg_sample_blocks(int32_t n, int32_t m) {
-  int64_t p = (kLrTargetCtas + n - 1) / n;
-  const int64_t most = (m + 4 * kLrSamples - 1) / (4 * kLrSamples);  // at least 16 samples per block
+// Sample rows in flight per thread: four, or two where the thread's slice is so wide (eight float4
+// per row) that four rows of it would not fit in registers beside z and the gradient.
+template <int VPT> struct LrSamples { static constexpr int value = VPT >= 8 ? 2 : 4; };
+// NS inner products travel as one vector (one shared-memory access).
+template <int NS> struct LrDots;
+template <> struct LrDots<4> { using type = float4; };
+template <> struct LrDots<2> { using type = float2; };
+__device__ __forceinline__ void dots_add(float4 &t, float4 v) { t.x += v.x; t.y += v.y; t.z += v.z; t.w += v.w; }
+__device__ __forceinline__ void dots_add(float2 &t, float2 v) { t.x += v.x; t.y += v.y; }
+__device__ __forceinline__ float4 dots_pack(const float (&d)[4]) { return make_float4(d[0], d[1], d[2], d[3]); }
+__device__ __forceinline__ float2 dots_pack(const float (&d)[2]) { return make_float2(d[0], d[1]); }
+__device__ __forceinline__ void dots_unpack(float4 v, float (&d)[4]) { d[0] = v.x; d[1] = v.y; d[2] = v.z; d[3] = v.w; }
+__device__ __forceinline__ void dots_unpack(float2 v, float (&d)[2]) { d[0] = v.x; d[1] = v.y; }
+
+// Column chunks (CTAs per cluster) for d columns: chunks of 4096 columns while a cluster of eight
+// covers the row, chunks of up to 8192 columns beyond that.
+static inline int32_t logreg_chunks(int64_t d) {
+  const int64_t half = (d + kLrHalfChunkCols - 1) / kLrHalfChunkCols;
+  return (int32_t)(half <= kLrMaxCluster ? half : (d + kLrChunkCols - 1) / kLrChunkCols);
+}
+
+static inline int32_t logreg_sample_blocks(int32_t n, int32_t m, int64_t d) {
+  const int64_t ctas_per_block = (int64_t)n * logreg_chunks(d);
+  int64_t p = (kLrTargetCtas + ctas_per_block - 1) / ctas_per_block;
+  const int64_t most = (m + 15) / 16;  // at least 16 samples per block
   if (p > most) p = most;
   if (p < 1) p = 1;
   return (int32_t)p;
@@ -55,7 +85,8 @@ struct LogregArgs {
   const float *A, *labels, *Z;
   float *partial;   // [n][P][d]
   int64_t d, ld;
-  int32_t n, m, P, samples_per_block;
+  int64_t chunk4;   // float4 column groups per CTA of a cluster (all of them when there is one CTA)
+  int32_t n, m, P, samples_per_block, chunks;
   float inv_m;
 };
 
@@ -63,13 +94,23 @@ __device__ __forceinline__ float dot4(float4 a, float4 b) {
   return fmaf(a.x, b.x, fmaf(a.y, b.y, fmaf(a.z, b.z, a.w * b.w)));
 }
 
-template <int VPT, int LOSS>
-__global__ void __launch_bounds__(kLrThreads) logreg_fused_kernel(const LogregArgs p) {
-  __shared__ float4 red[2][kLrWarps];
+// VPT float4 column groups per thread.  CLUSTER: launched as clusters of p.chunks CTAs along x; the
+// CTA of rank r takes the column groups [r * chunk4, (r + 1) * chunk4).
+template <int VPT, int LOSS, bool CLUSTER>
+__global__ void __launch_bounds__(kLrThreads, VPT == 1 ? 4 : VPT == 2 ? 3 : VPT == 4 ? 2 : 1)
+logreg_fused_kernel(const LogregArgs p) {
+  constexpr int NS = LrSamples<VPT>::value;
+  using Dots = typename LrDots<NS>::type;
+  __shared__ Dots red[2][kLrWarps];
+  __shared__ Dots share[2][kLrMaxCluster];   // the inner-product shares of the cluster's CTAs
+  namespace cg = cooperative_groups;
+  const int rank = CLUSTER ? (int)cg::this_cluster().block_rank() : 0;
   const int i = blockIdx.y;
-  const int blk = blockIdx.x;
+  const int blk = CLUSTER ? blockIdx.x / p.chunks : blockIdx.x;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int64_t d4 = p.d >> 2;
+  const int64_t cg0 = (int64_t)rank * p.chunk4;
+  const int64_t cg_end = min(d4, cg0 + p.chunk4);
   const int s_begin = blk * p.samples_per_block;
   const int s_end = min(p.m, s_begin + p.samples_per_block);
 
@@ -77,32 +118,34 @@ __global__ void __launch_bounds__(kLrThreads) logreg_fused_kernel(const LogregAr
   bool valid[VPT];
 #pragma unroll
   for (int j = 0; j < VPT; ++j) {
-    const int64_t cg = threadIdx.x + (int64_t)j * kLrThreads;
-    valid[j] = cg < d4;
-    z[j] = valid[j] ? *reinterpret_cast<const float4 *>(p.Z + (int64_t)i * p.ld + cg * 4)
+    const int64_t cgj = cg0 + threadIdx.x + (int64_t)j * kLrThreads;
+    valid[j] = cgj < cg_end;
+    z[j] = valid[j] ? *reinterpret_cast<const float4 *>(p.Z + (int64_t)i * p.ld + cgj * 4)
                     : make_float4(0.f, 0.f, 0.f, 0.f);
     acc[j] = make_float4(0.f, 0.f, 0.f, 0.f);
   }
-  const float *a_agent = p.A + (int64_t)i * p.m * p.d;
+  const float *a_agent = p.A + (int64_t)i * p.m * p.d + cg0 * 4;
   const float *l_agent = p.labels + (int64_t)i * p.m;
+  // every CTA of the cluster must be running before anybody writes into its shared memory
+  if (CLUSTER) cg::this_cluster().sync();
 
   int buf = 0;
-  for (int s = s_begin; s < s_end; s += kLrSamples) {
-    float4 a[kLrSamples][VPT];
-    float dot[kLrSamples];
+  for (int s = s_begin; s < s_end; s += NS) {
+    float4 a[NS][VPT];
+    float dot[NS];
 #pragma unroll
-    for (int jj = 0; jj < kLrSamples; ++jj) {
+    for (int jj = 0; jj < NS; ++jj) {
       const bool live = s + jj < s_end;
       const float *row = a_agent + (int64_t)(s + jj) * p.d;
 #pragma unroll
       for (int j = 0; j < VPT; ++j) {
-        const int64_t cg = threadIdx.x + (int64_t)j * kLrThreads;
-        a[jj][j] = (live && valid[j]) ? __ldcs(reinterpret_cast<const float4 *>(row + cg * 4))
+        const int64_t cgl = threadIdx.x + (int64_t)j * kLrThreads;   // column group inside the chunk
+        a[jj][j] = (live && valid[j]) ? __ldcs(reinterpret_cast<const float4 *>(row + cgl * 4))
                                       : make_float4(0.f, 0.f, 0.f, 0.f);
       }
     }
 #pragma unroll
-    for (int jj = 0; jj < kLrSamples; ++jj) {
+    for (int jj = 0; jj < NS; ++jj) {
       float t = 0.f;
 #pragma unroll
       for (int j = 0; j < VPT; ++j) t += dot4(a[jj][j], z[j]);
@@ -110,18 +153,26 @@ __global__ void __launch_bounds__(kLrThreads) logreg_fused_kernel(const LogregAr
       for (int o = 16; o > 0; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
       dot[jj] = t;
     }
-    if (lane == 0) red[buf][warp] = make_float4(dot[0], dot[1], dot[2], dot[3]);
+    if (lane == 0) red[buf][warp] = dots_pack(dot);
     __syncthreads();
-    float4 tot = red[buf][0];
+    Dots tot = red[buf][0];
 #pragma unroll
-    for (int w = 1; w < kLrWarps; ++w) {
-      const float4 v = red[buf][w];
-      tot.x += v.x; tot.y += v.y; tot.z += v.z; tot.w += v.w;
+    for (int w = 1; w < kLrWarps; ++w) dots_add(tot, red[buf][w]);
+    if (CLUSTER) {
+      // tot is this CTA's share (its column chunk).  Thread t hands it to the CTA of rank t;
+      // after the barrier every CTA adds the shares in rank order.  Two buffers: a CTA can only
+      // write the next iteration's shares after everybody has read those of the previous one.
+      cg::cluster_group cluster = cg::this_cluster();
+      if ((int)threadIdx.x < p.chunks) *cluster.map_shared_rank(&share[buf][rank], threadIdx.x) = tot;
+      cluster.sync();
+      tot = share[buf][0];
+      for (int r = 1; r < p.chunks; ++r) dots_add(tot, share[buf][r]);
     }
+    float margin[NS];
+    dots_unpack(tot, margin);
     buf ^= 1;  // the other buffer is free: everybody passed the barrier above after reading it
-    const float margin[kLrSamples] = {tot.x, tot.y, tot.z, tot.w};
 #pragma unroll
-    for (int jj = 0; jj < kLrSamples; ++jj) {
+    for (int jj = 0; jj < NS; ++jj) {
       float coef = 0.f;
       if (s + jj < s_end) {
         coef = sample_coef<LOSS>(__ldg(l_agent + s + jj), margin[jj], p.inv_m);
@@ -135,11 +186,11 @@ __global__ void __launch_bounds__(kLrThreads) logreg_fused_kernel(const LogregAr
       }
     }
   }
-  float *out = p.partial + ((int64_t)i * p.P + blk) * p.d;
+  float *out = p.partial + ((int64_t)i * p.P + blk) * p.d + cg0 * 4;
 #pragma unroll
   for (int j = 0; j < VPT; ++j) {
-    const int64_t cg = threadIdx.x + (int64_t)j * kLrThreads;
-    if (valid[j]) *reinterpret_cast<float4 *>(out + cg * 4) = acc[j];
+    const int64_t cgl = threadIdx.x + (int64_t)j * kLrThreads;
+    if (valid[j]) *reinterpret_cast<float4 *>(out + cgl * 4) = acc[j];
   }
 }
 
@@ -197,7 +248,7 @@ __global__ void __launch_bounds__(256) logreg_accum_kernel(const float *A, const
 static inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 size_t logreg_workspace_bytes(int32_t n, int32_t m, int64_t d) {
-  const size_t partial = (size_t)n * (size_t)logreg_sample_blocks(n, m) * (size_t)d * sizeof(float);
+  const size_t partial = (size_t)n * (size_t)logreg_sample_blocks(n, m, d) * (size_t)d * sizeof(float);
   const size_t coef = (size_t)n * (size_t)m * sizeof(float);
   return ((partial + 255) / 256) * 256 + ((coef + 255) / 256) * 256;
 }
@@ -209,11 +260,12 @@ template <int LOSS>
 static ceca_status_t enqueue_grad(const float *A, const float *targets, const float *Z, const float *noise, float *G,
                                   int32_t n, int32_t m, int64_t d, int64_t ld, void *scratch, cudaStream_t stream) {
   const float inv_m = (float)(1.0 / (double)m);
-  const int32_t P = logreg_sample_blocks(n, m);
+  const int32_t P = logreg_sample_blocks(n, m, d);
   float *partial = static_cast<float *>(scratch);
   const size_t partial_bytes = (((size_t)n * P * d * sizeof(float) + 255) / 256) * 256;
   float *coef = reinterpret_cast<float *>(static_cast<char *>(scratch) + partial_bytes);
-  const bool fast = (d % 4 == 0) && (ld % 4 == 0) && d <= (int64_t)kLrThreads * 4 * kLrMaxVpt && aligned16(A) &&
+  const int32_t chunks = logreg_chunks(d);
+  const bool fast = (d % 4 == 0) && (ld % 4 == 0) && chunks <= kLrMaxCluster && aligned16(A) &&
                     aligned16(Z) && aligned16(G) && (!noise || aligned16(noise)) && n <= 65535;
   if (fast) {
     LogregArgs a;
@@ -221,13 +273,30 @@ static ceca_status_t enqueue_grad(const float *A, const float *targets, const fl
     a.d = d; a.ld = ld; a.n = n; a.m = m; a.P = P;
     a.samples_per_block = (m + P - 1) / P;
     a.inv_m = inv_m;
-    const dim3 grid((unsigned)P, (unsigned)n);
-    const int64_t groups = (d / 4 + kLrThreads - 1) / kLrThreads;
-    if (groups <= 1)      logreg_fused_kernel<1, LOSS><<<grid, kLrThreads, 0, stream>>>(a);
-    else if (groups <= 2) logreg_fused_kernel<2, LOSS><<<grid, kLrThreads, 0, stream>>>(a);
-    else if (groups <= 4) logreg_fused_kernel<4, LOSS><<<grid, kLrThreads, 0, stream>>>(a);
-    else                  logreg_fused_kernel<8, LOSS><<<grid, kLrThreads, 0, stream>>>(a);
-    if (cudaGetLastError() != cudaSuccess) return CECA_ERR_CUDA;
+    a.chunks = chunks;
+    a.chunk4 = (d / 4 + chunks - 1) / chunks;
+    const int64_t groups = (a.chunk4 + kLrThreads - 1) / kLrThreads;   // float4 per thread and row
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)P * chunks, (unsigned)n);
+    cfg.blockDim = dim3(kLrThreads);
+    cfg.stream = stream;
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeClusterDimension;
+    attr.val.clusterDim.x = chunks; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
+    cudaError_t e;
+    if (chunks > 1) {
+      cfg.attrs = &attr; cfg.numAttrs = 1;
+      if (groups <= 1)      e = cudaLaunchKernelEx(&cfg, logreg_fused_kernel<1, LOSS, true>, a);
+      else if (groups <= 2) e = cudaLaunchKernelEx(&cfg, logreg_fused_kernel<2, LOSS, true>, a);
+      else if (groups <= 4) e = cudaLaunchKernelEx(&cfg, logreg_fused_kernel<4, LOSS, true>, a);
+      else                  e = cudaLaunchKernelEx(&cfg, logreg_fused_kernel<8, LOSS, true>, a);
+    } else {
+      if (groups <= 1)      e = cudaLaunchKernelEx(&cfg, logreg_fused_kernel<1, LOSS, false>, a);
+      else if (groups <= 2) e = cudaLaunchKernelEx(&cfg, logreg_fused_kernel<2, LOSS, false>, a);
+      else if (groups <= 4) e = cudaLaunchKernelEx(&cfg, logreg_fused_kernel<4, LOSS, false>, a);
+      else                  e = cudaLaunchKernelEx(&cfg, logreg_fused_kernel<8, LOSS, false>, a);
+    }
+    if (e != cudaSuccess) return CECA_ERR_CUDA;
     const int64_t work = (int64_t)n * (d / 4);
     logreg_reduce_kernel<<<(unsigned)((work + 255) / 256), 256, 0, stream>>>(partial, noise, G, n, P, d, ld);
     return cudaGetLastError() == cudaSuccess ? CECA_OK : CECA_ERR_CUDA;

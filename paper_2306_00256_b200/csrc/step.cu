@@ -249,22 +249,41 @@ static cudaError_t enqueue_step_as(const Plan &plan, const TXY *X, const TXY *Y,
   const bool has_g = (G != nullptr);
   const int ymode = Yo ? (plan.reads_y ? 1 : 0) : ((Y && plan.reads_y) ? 3 : 2);
   const bool use_y = (ymode == 1 || ymode == 3);
-  constexpr size_t kAlignXY = VW * sizeof(TXY), kAlignG = VW * sizeof(TG);
-  const bool vec_ok = (ld % VW == 0) && aligned_to(X, kAlignXY) && aligned_to(Xo, kAlignXY) &&
-                      (!Yo || aligned_to(Yo, kAlignXY)) && (!use_y || aligned_to(Y, kAlignXY)) &&
-                      (!has_g || aligned_to(G, kAlignG));
-  const int64_t d_vec = vec_ok ? (d / VW) * VW : 0;  // columns covered by vector accesses
+  // Vector accesses need every row of every array to start on a VW-element boundary once the first
+  // `head` columns are set aside: ld a multiple of VW, and all base pointers off such a boundary by
+  // the same number of elements (zero for buffers that come straight from an allocator; the same
+  // non-zero amount for, say, views that skip the first k elements of aligned buffers).  The head
+  // and the ragged tail (fewer than VW columns each) run the scalar form.
+  auto misalign = [](const void *ptr, size_t elem) { return (int64_t)((reinterpret_cast<uintptr_t>(ptr) / elem) % VW); };
+  const int64_t mis = misalign(X, sizeof(TXY));
+  const bool vec_ok = (ld % VW == 0) && aligned_to(X, sizeof(TXY)) && misalign(Xo, sizeof(TXY)) == mis &&
+                      aligned_to(Xo, sizeof(TXY)) && (!Yo || (misalign(Yo, sizeof(TXY)) == mis && aligned_to(Yo, sizeof(TXY)))) &&
+                      (!use_y || (misalign(Y, sizeof(TXY)) == mis && aligned_to(Y, sizeof(TXY)))) &&
+                      (!has_g || (misalign(G, sizeof(TG)) == mis && aligned_to(G, sizeof(TG))));
+  int64_t head = vec_ok ? (VW - mis) % VW : 0;   // scalar columns in front of the vector body
+  if (head > d) head = d;
+  const int64_t d_vec = vec_ok ? ((d - head) / VW) * VW : 0;  // columns covered by vector accesses
+  auto shifted = [&](const StepArgs &from, int64_t c0, int64_t count) {
+    StepArgs t = from;
+    t.X = X + c0; t.Xo = Xo + c0; t.Yo = Yo ? Yo + c0 : nullptr;
+    t.Y = Y ? Y + c0 : nullptr;
+    t.G = G ? G + c0 : nullptr;
+    t.ncolv = count;
+    return t;
+  };
   if (d_vec > 0) {
-    a.ncolv = d_vec / VW;
-    cudaError_t e = launch_walk<V, TXY, TG, Y_FORMS, ALLOW_NO_G>(a, has_g, ymode, stream);
+    const StepArgs body = shifted(a, head, d_vec / VW);
+    cudaError_t e = launch_walk<V, TXY, TG, Y_FORMS, ALLOW_NO_G>(body, has_g, ymode, stream);
     if (e != cudaSuccess) return e;
   }
-  if (d_vec < d) {  // ragged tail (or everything, when rows are not aligned for vector accesses)
-    StepArgs t = a;
-    t.X = X + d_vec; t.Xo = Xo + d_vec; t.Yo = Yo ? Yo + d_vec : nullptr;
-    t.Y = Y ? Y + d_vec : nullptr;
-    t.G = G ? G + d_vec : nullptr;
-    t.ncolv = d - d_vec;
+  if (d_vec == 0) head = 0;   // no vector body: one scalar launch covers everything
+  if (head > 0) {
+    const StepArgs t = shifted(a, 0, head);
+    cudaError_t e = launch_walk<float, TXY, TG, Y_FORMS, ALLOW_NO_G>(t, has_g, ymode, stream);
+    if (e != cudaSuccess) return e;
+  }
+  if (head + d_vec < d) {  // ragged tail (or everything, when rows cannot be aligned for vector accesses)
+    const StepArgs t = shifted(a, head + d_vec, d - head - d_vec);
     cudaError_t e = launch_walk<float, TXY, TG, Y_FORMS, ALLOW_NO_G>(t, has_g, ymode, stream);
     if (e != cudaSuccess) return e;
   }

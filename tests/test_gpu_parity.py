@@ -136,6 +136,7 @@ def test_step_with_more_cycles_than_one_grid_dimension_holds():
 
 
 @pytest.mark.parametrize("n,d,ld,offset", [(6, 37, 40, 0), (6, 37, 41, 0), (24, 1000, 1024, 4), (24, 1000, 1024, 1),
+                                           (24, 1000, 1024, 2), (24, 1003, 1024, 3), (5, 2, 8, 3), (5, 3, 8, 1), (5, 7, 8, 2),
                                            (97, 513, 517, 3), (100, 4096, 4100, 0)])
 def test_step_padded_rows_and_unaligned_bases(n, d, ld, offset):
     x, y, g = synth.step_inputs(n, d, seed=7, x_std=1.0, g_std=0.5, same_xy=False)
@@ -154,6 +155,24 @@ def test_step_padded_rows_and_unaligned_bases(n, d, ld, offset):
                 assert torch.isnan(xob[offset:offset + n * ld].view(n, ld)[:, d:]).all()
                 assert torch.isnan(yob[offset:offset + n * ld].view(n, ld)[:, d:]).all()
             assert torch.isnan(xob[:offset]).all() and torch.isnan(xob[offset + n * ld:]).all()
+
+
+def test_step_with_differently_misaligned_arrays():
+    """X, Y, G and the outputs each start a different number of elements off a 16-byte boundary: no common
+    scalar head exists, every column runs the scalar form, and the result is the same."""
+    n, d, ld, gamma = 24, 1000, 1024, 0.25
+    x, y, g = synth.step_inputs(n, d, seed=11, x_std=1.0, g_std=0.5, same_xy=False)
+    for variant in _variants(n):
+        for k in range(_tau(n)):
+            (X, _), (Y, _), (G, _) = _put(x.to(DEV), ld, 1), _put(y.to(DEV), ld, 2), _put(g.to(DEV), ld, 3)
+            (Xo, xob), (Yo, yob) = _padded(n, d, ld, 0), _padded(n, d, ld, 5)
+            ceca.ceca_gossip_sgd_step(X, Y, G, gamma, variant, k, X_out=Xo, Y_out=Yo)
+            want_x, want_y = oracle.step(_np(x), _np(y), _np(g), np.float32(gamma), variant, k)
+            tol = STEP_TOL * _scale(gamma, (x, 1), (y, 1), (g, gamma))
+            assert np.abs(_np(Xo) - want_x).max() <= tol
+            assert np.abs(_np(Yo) - want_y).max() <= tol
+            assert torch.isnan(yob[:5]).all() and torch.isnan(yob[5 + n * ld:]).all()
+            assert torch.isnan(xob[n * ld:]).all()
 
 
 def test_step_without_gradient_is_a_ceca_round_and_y_may_be_absent_in_round_zero():
@@ -529,7 +548,9 @@ def _grad_tol(d, want):
 
 
 @pytest.mark.parametrize("n,m,d", [(5, 100, 32), (6, 100, 32), (3, 37, 4096), (2, 50, 8192), (2, 33, 1028),
-                                   (4, 16, 2048), (3, 20, 30), (2, 9, 8200), (1, 5, 1), (7, 1, 64)])
+                                   (4, 16, 2048), (3, 20, 30), (2, 9, 8200), (1, 5, 1), (7, 1, 64),
+                                   # wider than one CTA's registers: clusters of 2 to 8 CTAs, one column chunk each
+                                   (2, 21, 4100), (2, 21, 8196), (3, 37, 16384), (1, 18, 40000), (2, 33, 65536), (2, 5, 65540), (2, 4, 70000)])
 def test_logreg_grad_matches_oracle(n, m, d):
     a, lab, x_star = synth.logreg_problem(n, m, d, seed=n + m + d, flip=0.1, hetero_std=0.5)
     gen = torch.Generator().manual_seed(1)
@@ -548,7 +569,7 @@ def test_logreg_grad_matches_oracle(n, m, d):
             assert torch.equal(G, G2)  # run-to-run identical
 
 
-@pytest.mark.parametrize("n,m,d,ld", [(6, 40, 512, 516), (6, 40, 512, 513), (3, 33, 2052, 2080), (5, 50, 10, 12)])
+@pytest.mark.parametrize("n,m,d,ld", [(6, 40, 512, 516), (6, 40, 512, 513), (3, 33, 2052, 2080), (5, 50, 10, 12), (2, 9, 12288, 12292)])
 def test_gradients_with_padded_rows_leave_padding_and_workspace_guard_alone(n, m, d, ld):
     """X, Y, G (and the least-squares noise) with ld > d; the columns between d and ld of G, and a guard
     area behind the stated workspace size, must keep their canary values."""
@@ -655,7 +676,7 @@ def _lsq_tol(a, b, z):
     return 4 * u * (np.sqrt(d) + np.sqrt(m)) * s + 1e-7
 
 
-@pytest.mark.parametrize("n,m,d", [(258, 50, 10), (6, 50, 10), (4, 64, 2048), (3, 37, 4096), (5, 20, 12), (2, 7, 1)])
+@pytest.mark.parametrize("n,m,d", [(258, 50, 10), (6, 50, 10), (4, 64, 2048), (3, 37, 4096), (5, 20, 12), (2, 7, 1), (2, 30, 16384)])
 def test_lsq_grad_matches_oracle(n, m, d):
     a, b, _ = synth.lsq_problem(n, m, d, seed=n + d, sigma_s=0.1)
     gen = torch.Generator().manual_seed(3)
@@ -848,7 +869,8 @@ def _bf16_tol(want, scale, xy_bf16):
 
 @pytest.mark.parametrize("xy_bf16", [False, True])
 @pytest.mark.parametrize("n,d,ld,offset", [(1, 9, 9, 0), (5, 37, 37, 0), (6, 64, 64, 0), (24, 1000, 1000, 0), (24, 1000, 1008, 8),
-                                            (24, 1001, 1004, 4), (97, 4100, 4104, 0), (100, 70001, 70008, 0)])
+                                            (24, 1001, 1004, 4), (24, 1000, 1008, 3), (24, 1001, 1008, 5), (6, 5, 8, 6),
+                                            (97, 4100, 4104, 0), (100, 70001, 70008, 0)])
 def test_step_with_bf16_storage_matches_oracle(xy_bf16, n, d, ld, offset):
     gamma = 0.1
     x, y, g = synth.step_inputs(n, d, seed=n + d, x_std=1.0, g_std=1.0, same_xy=False)
