@@ -66,7 +66,7 @@ WORKLOADS = {
     "consensus_fused_1026_smem": dict(kind="consensus", n=1026, d=1 << 18, variant=2, fused=2),
     "consensus_rounds_1026": dict(kind="consensus", n=1026, d=1 << 18, variant=2, fused=0),
     "logreg_grad": dict(kind="logreg", n=63, m=2000, d=4096, variant=2, gamma=0.01),
-    # wider models at the same 2 GB of samples: clusters of 2 (d = 8192) and 8 (d = 32768) CTAs, 4096 columns each
+    # wider models at the same 2 GB of samples: eight float4 per thread (d = 8192), clusters of 8 CTAs of 4096 columns (d = 32768)
     "logreg_grad_d8192": dict(kind="logreg", n=32, m=2000, d=8192, variant=2, gamma=0.01),
     "logreg_grad_d32768": dict(kind="logreg", n=8, m=2000, d=32768, variant=2, gamma=0.01),
     # whole iterations (gradient kernel + fused step), one CECA cycle captured in a CUDA graph and replayed

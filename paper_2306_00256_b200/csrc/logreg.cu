@@ -55,9 +55,12 @@ __device__ __forceinline__ float2 dots_pack(const float (&d)[2]) { return make_f
 __device__ __forceinline__ void dots_unpack(float4 v, float (&d)[4]) { d[0] = v.x; d[1] = v.y; d[2] = v.z; d[3] = v.w; }
 __device__ __forceinline__ void dots_unpack(float2 v, float (&d)[2]) { d[0] = v.x; d[1] = v.y; }
 
-// Column chunks (CTAs per cluster) for d columns: chunks of 4096 columns while a cluster of eight
-// covers the row, chunks of up to 8192 columns beyond that.
+// Column chunks (CTAs per cluster) for d columns.  One CTA while its registers hold the row
+// (d <= 8192: a cluster barrier per batch of rows costs more than the narrower slices win, 0.74
+// against 0.66 of the copy rate at d = 8192); beyond that chunks of 4096 columns (two CTAs per SM,
+// four rows in flight) while a cluster of eight covers the row, chunks of up to 8192 columns above.
 static inline int32_t logreg_chunks(int64_t d) {
+  if (d <= kLrChunkCols) return 1;
   const int64_t half = (d + kLrHalfChunkCols - 1) / kLrHalfChunkCols;
   return (int32_t)(half <= kLrMaxCluster ? half : (d + kLrChunkCols - 1) / kLrChunkCols);
 }
