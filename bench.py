@@ -85,12 +85,20 @@ FALLBACK_HBM_GBS = 6650.0
 # file when the counters were taken).  A kernel source that has changed since makes the entry stale
 # and `traffic` is reported as null until the capture is redone.
 NCU_TRAFFIC = {
-    # 19.76 B per agent-parameter measured on step_small (2.5166 GB read + 1.6263 GB written for
+    # 19.73 B per agent-parameter measured on step_small (2.5166 GB read + 1.6220 GB written for
     # 100 x 2,097,152 units); traffic is proportional to the units, scaled to n*d of resnet50_step
-    "step_small": (4.143e9, "step_walk_kernel__step_small__ncu_full.md", "step.cu", "955600f7f709"),
-    "resnet50_step": (19.755 * 100 * 25_557_032, "step_walk_kernel__step_small__ncu_full.md", "step.cu", "955600f7f709"),
-    "consensus_rounds": (10.56e9, "step_walk_kernel__consensus_rounds_n97_d1M__dram.md", "step.cu", "955600f7f709"),
-    "logreg_grad": (2.0736e9 + 29.9e6, "logreg_fused_kernel__n63_m2000_d4096__ncu_full.md", "logreg.cu", "e8cef610359e"),
+    "step_small": (4.1386e9, "dram_traffic__step_consensus_gradient.md", "step.cu", "b16a43e291d9"),
+    "resnet50_step": (19.734 * 100 * 25_557_032, "dram_traffic__step_consensus_gradient.md", "step.cu", "b16a43e291d9"),
+    # seven launches of a cycle: round 0 moves 1.168 GB, the six others 1.565 GB each
+    "consensus_rounds": (10.558e9, "dram_traffic__step_consensus_gradient.md", "step.cu", "b16a43e291d9"),
+    # fused kernel 2.0735 GB + fixed-order reduce 0.0299 GB
+    "logreg_grad": (2.1034e9, "dram_traffic__step_consensus_gradient.md", "logreg.cu", "b3cedf2f4e6b"),
+    "logreg_grad_d32768": (2.1357e9, "dram_traffic__step_consensus_gradient.md", "logreg.cu", "b3cedf2f4e6b"),
+    # register-block kernel: captured at d = 2^19 (0.5522 GB per launch) and doubled for d = 2^20 (traffic is per tile)
+    "consensus_fused_small": (0.5522e9, "consensus_block_kernel__n97_n258_n1026__ncu_full.md", "consensus_block.cu", "c9a9e499f644"),
+    "consensus_fused": (1.1044e9, "consensus_block_kernel__n97_n258_n1026__ncu_full.md", "consensus_block.cu", "c9a9e499f644"),
+    "consensus_fused_258": (1.5641e9, "consensus_block_kernel__n97_n258_n1026__ncu_full.md", "consensus_block.cu", "c9a9e499f644"),
+    "consensus_fused_1026": (3.1769e9, "consensus_block_kernel__n97_n258_n1026__ncu_full.md", "consensus_block.cu", "c9a9e499f644"),
 }
 
 

@@ -100,6 +100,11 @@ ceca_status_t ceca_schedule(int32_t n, ceca_variant_t variant, int64_t k, ceca_r
  * given) skips that write: 16 bytes per agent-parameter; the caller's Y buffer keeps its old contents
  * until round 0 overwrites it.  Y_out == NULL with Y given in any other round is CECA_ERR_INVALID_ARG.
  * fp32 arithmetic; a, b and 1-a, 1-b are formed in fp64 on the host and rounded once.
+ * Speed: 128-bit accesses need ld % 4 == 0 and every array (X, Y, G, X_out, Y_out) starting the same
+ * number of floats past a 16-byte boundary -- zero for whole allocations, or a common offset for
+ * views that skip the same number of leading elements; up to three leading and three trailing
+ * columns then run as a second, scalar launch.  Any other layout is correct too, but runs the scalar
+ * form for every column (about 0.84 of the full rate).
  */
 ceca_status_t ceca_gossip_sgd_step(const float *X, const float *Y, const float *G, float *X_out,
                                    float *Y_out, int32_t n, int64_t d, int64_t ld, float gamma,
@@ -181,6 +186,9 @@ ceca_status_t ceca_consensus_rounds(const float *X, const float *Y, float *X_out
  * workspace: device, at least ceca_workspace_bytes(CECA_WS_LOGREG_GRAD, n, m, d) bytes; holds
  * per-block partial sums that a second, fixed-order pass adds up, so results are identical from
  * run to run.
+ * Speed: A is read once when d % 4 == 0, ld % 4 == 0, d <= 65536 and A, X / Y, G are 16-byte aligned
+ * (above d = 8192 the kernel runs as thread-block clusters, one column chunk per CTA); any other
+ * shape is correct too but reads A twice.
  */
 ceca_status_t dsgd_logreg_grad(const float *A, const float *labels, const float *X, const float *Y,
                                int64_t k, float *G, int32_t n, int32_t m, int64_t d, int64_t ld,
@@ -290,6 +298,10 @@ ceca_status_t ceca_fused_wait_selftest(const float *X, float *X_out, int32_t n, 
  * copies and the kernels of neighbouring slabs overlapping on internal streams.
  * workspace: DEVICE memory, workspace_bytes >= ceca_workspace_bytes(CECA_WS_STEP_HOST, n, 0, d);
  * more workspace means wider slabs.  The call returns after all slabs have been written back.
+ * It takes no stream: the copies and kernels run on three internal non-blocking streams that are
+ * created and destroyed inside the call and are ordered after nothing of the caller's.  Device work
+ * of the caller that still reads or writes `workspace` (a pending kernel or memset on any stream)
+ * must therefore have finished before the call; the host buffers must not be in use by pending copies.
  */
 ceca_status_t ceca_gossip_sgd_step_host(float *X, float *Y, const float *G, int32_t n, int64_t d,
                                         int64_t ld, float gamma, ceca_variant_t variant, int64_t k,
