@@ -89,6 +89,8 @@ NCU_TRAFFIC = {
     # 100 x 2,097,152 units); traffic is proportional to the units, scaled to n*d of resnet50_step
     "step_small": (4.1386e9, "dram_traffic__step_consensus_gradient.md", "step.cu", "b16a43e291d9"),
     "resnet50_step": (19.734 * 100 * 25_557_032, "dram_traffic__step_consensus_gradient.md", "step.cu", "b16a43e291d9"),
+    # cycles of two rows (every CECA-1P round): 19.72 B per agent-parameter on step_small's round 6, scaled by units
+    "resnet18_step": (19.72 * 24 * 11_689_512, "dram_traffic__step_consensus_gradient.md", "step.cu", "b16a43e291d9"),
     # seven launches of a cycle: round 0 moves 1.168 GB, the six others 1.565 GB each
     "consensus_rounds": (10.558e9, "dram_traffic__step_consensus_gradient.md", "step.cu", "b16a43e291d9"),
     # fused kernel 2.0735 GB + fixed-order reduce 0.0299 GB
