@@ -68,6 +68,7 @@ WORKLOADS = {
     "logreg_grad": dict(kind="logreg", n=63, m=2000, d=4096, variant=2, gamma=0.01),
     # wider models at the same 2 GB of samples: eight float4 per thread (d = 8192), clusters of 8 CTAs of 4096 columns (d = 32768)
     "logreg_grad_d8192": dict(kind="logreg", n=32, m=2000, d=8192, variant=2, gamma=0.01),
+    "logreg_grad_d16384": dict(kind="logreg", n=16, m=2000, d=16384, variant=2, gamma=0.01),
     "logreg_grad_d32768": dict(kind="logreg", n=8, m=2000, d=32768, variant=2, gamma=0.01),
     # whole iterations (gradient kernel + fused step), one CECA cycle captured in a CUDA graph and replayed
     "logreg_train": dict(kind="train", n=63, m=2000, d=4096, variant=2, gamma=0.01, loss="logistic"),

@@ -246,6 +246,9 @@ ceca_status_t dsgd_grad_shard_apply(const float *A_shard, const float *targets, 
  *     rejected with CECA_ERR_STATIC_SCRATCH before anything is launched.
  *   - The first call on each device looks up the buffer's device address (with that device
  *     current); make that first call ordinary eager work, before any stream capture is begun.
+ *     The address is remembered per device ordinal for the life of the process: it does not
+ *     survive cudaDeviceReset or the destruction of the device's primary context, after which
+ *     this entry point must not be used again in the same process.
  *   - All calls on a device share the one buffer.  Nothing in it needs clearing between calls
  *     (each call overwrites what it later reads), but two calls that may run on the GPU at the
  *     same time -- different streams, or different host threads -- race on it: order them.
