@@ -86,6 +86,7 @@ struct BlockArgs {
   int32_t boxes, box_rows;   // a tile lands as `boxes` TMA boxes of `box_rows` rows (boxes * box_rows >= n)
   uint32_t tile_bytes; // shared-memory footprint of one tile (a multiple of 128 that holds blocks * CB rows and all boxes)
   int32_t single_xch;  // one exchange tile instead of two (saves shared memory, costs a second barrier per round)
+  int32_t tma_out;     // results leave through the exchange tiles and TMA tensor stores instead of register stores
   int32_t wait_polls;
   uint32_t tx_bytes;   // bytes the landing barrier is armed for
   float outI, outJ;
@@ -256,10 +257,12 @@ __device__ __forceinline__ void dispatch_round(int sel, int s, int n, pk2 (&Ih)[
 template <int CB, int LPB, int MAXT>
 __global__ void __launch_bounds__(MAXT, 1)
 consensus_block_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_y,
+                       const __grid_constant__ CUtensorMap map_xo, const __grid_constant__ CUtensorMap map_yo,
                        const __grid_constant__ BlockArgs p) {
   constexpr int kTileCols = 2 * LPB;
   constexpr int RB = kTileCols * (int)sizeof(float);
   constexpr bool kBalanced = LPB >= 16;
+  constexpr bool kTmaOut = LPB < 32;   // the TMA-store form exists for the narrow tiles only (a launch parameter picks it)
   // received rows in flight per thread: eight, or four where the state leaves fewer than 36 other registers
   constexpr int kInFlight = 65536 / MAXT - 4 * CB >= 36 ? 8 : 4;
   extern __shared__ __align__(128) unsigned char smem_raw[];
@@ -315,9 +318,11 @@ consensus_block_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
       // that it cannot write into shared memory of a finished CTA) and give up without storing.
       if (threadIdx.x == 0) atomicExch(p.status, 1);
       mbar_wait_bounded(&bar, phase, (uint32_t)p.wait_polls);
+      if (kTmaOut && threadIdx.x == 0) tma_store_wait_read();   // an earlier tile's stores still read shared memory
       return;
     }
     phase ^= 1u;
+    bool staging_free = false;   // TMA-store form: the previous tile's stores have finished reading the exchange tiles
 
     pk2 Ih[CB], Jh[CB];
     {
@@ -366,6 +371,12 @@ consensus_block_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
         // the first round's neighbours) are done: the next tile may land while this one is finished
         issue_load(next_tile);
       }
+      if (kTmaOut && p.tma_out && rnd == 1) {
+        // the first publish of this tile: the previous tile's TMA stores must be done with the exchange tiles
+        if (threadIdx.x == 0) tma_store_wait_read();
+        __syncthreads();
+        staging_free = true;
+      }
       // The first round finds every row's payload in the landed tile and publishes nothing.
       q.publish = rnd > 0;
       const uint32_t buf_tile = rnd == 0 ? ((mode & kBkPayloadJ) ? y_tile : 0u) : ((rnd & 1) || p.single_xch ? 1u : 2u);
@@ -379,8 +390,36 @@ consensus_block_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
     }
 
     const int32_t col = tile * kTileCols + 2 * lane;
-    // surplus threads (only where a block is narrower than a warp) shadow the last block and write nothing
-    if (LPB < 32 && (int)(threadIdx.x / LPB) >= p.blocks) {
+    if (kTmaOut && p.tma_out) {
+      // Results go into the two exchange tiles (X+ into the first, Y+ into the second) and leave as TMA
+      // tensor stores, which clip at row n and column d.  The CTA does not wait for them: they drain
+      // while the next tile lands and runs its first round, which touches neither exchange tile.
+      if (!staging_free && threadIdx.x == 0) tma_store_wait_read();
+      __syncthreads();   // the last round's reads of the exchange tiles are done (and the old stores, see above)
+      const pk2 oI = pk_make(p.outI, p.outI), oJ = pk_make(p.outJ, p.outJ);
+      const uint32_t sx = sm_land_x + p.tile_bytes + own_off, sy = sx + p.tile_bytes;
+      static_for<CB>([&](auto J) {
+        constexpr int j = CECA_IDX(J);
+        if (!kBalanced || j < CB - 1 || q.full) sts64<j * RB>(sx, mul2(oI, Ih[j]));
+      });
+      if (p.has_y_out) {
+        static_for<CB>([&](auto J) {
+          constexpr int j = CECA_IDX(J);
+          if (!kBalanced || j < CB - 1 || q.full) sts64<j * RB>(sy, mul2(oJ, Jh[j]));
+        });
+      }
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic writes -> visible to the TMA unit
+      __syncthreads();
+      if (threadIdx.x == 0) {
+        for (int b = 0; b < p.boxes; ++b) {
+          const int row0 = b * p.box_rows;
+          tma_store_2d(&map_xo, tile * kTileCols, row0, smem_raw + p.tile_bytes + (size_t)row0 * RB);
+          if (p.has_y_out) tma_store_2d(&map_yo, tile * kTileCols, row0, smem_raw + 2 * (size_t)p.tile_bytes + (size_t)row0 * RB);
+        }
+        tma_store_commit();
+      }
+    } else if (LPB < 32 && (int)(threadIdx.x / LPB) >= p.blocks) {
+      // surplus threads (only where a block is narrower than a warp) shadow the last block and write nothing
     } else if (col + 1 < p.d) {
       const pk2 oI = pk_make(p.outI, p.outI), oJ = pk_make(p.outJ, p.outJ);
       float *dst = p.Xo + (int64_t)q.i0 * p.ld + col;
@@ -418,6 +457,7 @@ consensus_block_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
       if (threadIdx.x == 0) issue_load(next_tile);
     }
   }
+  if (kTmaOut && p.tma_out && threadIdx.x == 0) tma_store_wait_read();   // shared memory must outlive the stores' reads
 }
 
 // ---- host side ----------------------------------------------------------------------------------
@@ -497,13 +537,14 @@ bool consensus_block_supports(int32_t n, ceca_variant_t variant, int32_t rounds,
 
 // Register budgets by block size (the state takes 4 * CB registers): a roomy one, and a lean one that
 // still compiles without spilling to speak of.  65536 / kMaxThreads registers per thread.
+constexpr int kBkTmaOutMaxCtas = 2;
 template <int CB> struct BlockRegs {
   static constexpr int kRoomy = CB >= 15 ? 384 : CB >= 11 ? 640 : CB >= 7 ? 768 : 1024;
   static constexpr int kLean = CB >= 15 ? 512 : CB >= 11 ? 768 : 1024;
 };
 
 template <int CB, int LPB, int MAXT>
-static cudaError_t launch_block_regs(const CUtensorMap &mx, const CUtensorMap &my, const BlockArgs &a, int threads,
+static cudaError_t launch_block_regs(const CUtensorMap *maps, const BlockArgs &a, int threads,
                                      size_t smem, int *per_sm_out, bool launch, cudaStream_t stream) {
   static std::atomic<uint64_t> attr_done{0};
   cudaError_t e = set_max_shared_once(reinterpret_cast<const void *>(consensus_block_kernel<CB, LPB, MAXT>),
@@ -520,13 +561,12 @@ static cudaError_t launch_block_regs(const CUtensorMap &mx, const CUtensorMap &m
   // persistent CTAs: as many as fit on the device at once, not more than there are tiles
   const int64_t resident = (int64_t)sms * per_sm;
   const int grid = (int)(a.tiles < resident ? a.tiles : resident);
-  consensus_block_kernel<CB, LPB, MAXT><<<grid, threads, smem, stream>>>(mx, my, a);
+  consensus_block_kernel<CB, LPB, MAXT><<<grid, threads, smem, stream>>>(maps[0], maps[1], maps[2], maps[3], a);
   return cudaGetLastError();
 }
 
 template <int CB, int LPB>
-static cudaError_t launch_block(const CUtensorMap &mx, const CUtensorMap &my, BlockArgs &a, int threads, int cmin,
-                                cudaStream_t stream) {
+static cudaError_t launch_block(const CUtensorMap *maps, BlockArgs &a, int threads, int cmin, cudaStream_t stream) {
   for (int t = 0; t < a.rounds; ++t) {
     BlockRound &r = a.rd[t];
     const int pay = (r.mode & kBkPayloadJ) ? 1 : 0;
@@ -542,11 +582,11 @@ static cudaError_t launch_block(const CUtensorMap &mx, const CUtensorMap &my, Bl
     if (smem > kBkSmemLimit) continue;
     int roomy = 0, lean = 0;
     if (threads <= kRoomy) {
-      cudaError_t e = launch_block_regs<CB, LPB, kRoomy>(mx, my, a, threads, smem, &roomy, false, stream);
+      cudaError_t e = launch_block_regs<CB, LPB, kRoomy>(maps, a, threads, smem, &roomy, false, stream);
       if (e != cudaSuccess) return e;
     }
     if (kLean != kRoomy && threads <= kLean) {
-      cudaError_t e = launch_block_regs<CB, LPB, kLean>(mx, my, a, threads, smem, &lean, false, stream);
+      cudaError_t e = launch_block_regs<CB, LPB, kLean>(maps, a, threads, smem, &lean, false, stream);
       if (e != cudaSuccess) return e;
     }
     if (roomy > best) { best = roomy; best_single = single; best_lean = 0; }
@@ -554,10 +594,14 @@ static cudaError_t launch_block(const CUtensorMap &mx, const CUtensorMap &my, Bl
   }
   if (best < 1) return cudaErrorInvalidConfiguration;
   a.single_xch = best_single;
+  // Narrow tiles with both exchange tiles and at most kBkTmaOutMaxCtas CTAs per SM: register stores would hold
+  // the whole CTA (and with it the SM) until the memory system has taken them; TMA stores from the
+  // exchange tiles let the next tile start meanwhile.
+  a.tma_out = (LPB < 32 && !best_single && best <= kBkTmaOutMaxCtas) ? 1 : 0;
   const size_t smem = ((a.has_y_in ? 2 : 1) + (best_single ? 1 : 2)) * tile_bytes;
   int per_sm = 0;
-  if (best_lean) return launch_block_regs<CB, LPB, kLean>(mx, my, a, threads, smem, &per_sm, true, stream);
-  return launch_block_regs<CB, LPB, kRoomy>(mx, my, a, threads, smem, &per_sm, true, stream);
+  if (best_lean) return launch_block_regs<CB, LPB, kLean>(maps, a, threads, smem, &per_sm, true, stream);
+  return launch_block_regs<CB, LPB, kRoomy>(maps, a, threads, smem, &per_sm, true, stream);
 }
 
 // Arguments are assumed validated by the caller (shapes, aliasing, 16-byte alignment of X / Y and
@@ -609,14 +653,16 @@ ceca_status_t consensus_block(const float *X, const float *Y, float *Xo, float *
   // a box counts in full towards the barrier, rows and columns outside the matrix included
   a.tx_bytes = (uint32_t)t.boxes * t.box_rows * tile_cols * sizeof(float) * (a.has_y_in ? 2u : 1u) + tx_extra;
 
-  CUtensorMap mx, my;
-  if (!tensor_map_2d(&mx, X, n, d, ld, tile_cols, t.box_rows)) return CECA_ERR_CUDA;
-  if (!tensor_map_2d(&my, a.has_y_in ? Y : X, n, d, ld, tile_cols, t.box_rows)) return CECA_ERR_CUDA;
+  CUtensorMap maps[4];   // X in, Y in, X out, Y out (unused ones alias a used one)
+  if (!tensor_map_2d(&maps[0], X, n, d, ld, tile_cols, t.box_rows)) return CECA_ERR_CUDA;
+  if (!tensor_map_2d(&maps[1], a.has_y_in ? Y : X, n, d, ld, tile_cols, t.box_rows)) return CECA_ERR_CUDA;
+  if (!tensor_map_2d(&maps[2], Xo, n, d, ld, tile_cols, t.box_rows)) return CECA_ERR_CUDA;
+  if (!tensor_map_2d(&maps[3], Yo ? Yo : Xo, n, d, ld, tile_cols, t.box_rows)) return CECA_ERR_CUDA;
 
   cudaError_t e = cudaErrorInvalidConfiguration;
   if (g.lpb == 32) {
     switch (g.cb) {
-#define CECA_BK_LAUNCH(CB) case CB: e = launch_block<CB, 32>(mx, my, a, g.threads, g.cmin, stream); break;
+#define CECA_BK_LAUNCH(CB) case CB: e = launch_block<CB, 32>(maps, a, g.threads, g.cmin, stream); break;
       CECA_BK_LAUNCH(1) CECA_BK_LAUNCH(2) CECA_BK_LAUNCH(3) CECA_BK_LAUNCH(4) CECA_BK_LAUNCH(5) CECA_BK_LAUNCH(6)
       CECA_BK_LAUNCH(7) CECA_BK_LAUNCH(8) CECA_BK_LAUNCH(9) CECA_BK_LAUNCH(10) CECA_BK_LAUNCH(11) CECA_BK_LAUNCH(12)
       CECA_BK_LAUNCH(13) CECA_BK_LAUNCH(14) CECA_BK_LAUNCH(15) CECA_BK_LAUNCH(16) CECA_BK_LAUNCH(17) CECA_BK_LAUNCH(18)
@@ -626,7 +672,7 @@ ceca_status_t consensus_block(const float *X, const float *Y, float *Xo, float *
       default: break;
     }
   } else if (g.lpb == 16) {
-#define CECA_BK_LAUNCH(CB) case CB: e = launch_block<CB, 16>(mx, my, a, g.threads, g.cmin, stream); break;
+#define CECA_BK_LAUNCH(CB) case CB: e = launch_block<CB, 16>(maps, a, g.threads, g.cmin, stream); break;
     switch (g.cb) {   // n = 257 .. 512 in 16, 24 or 32 blocks: 15 to 21 agents per block
       CECA_BK_LAUNCH(15) CECA_BK_LAUNCH(16) CECA_BK_LAUNCH(17) CECA_BK_LAUNCH(18) CECA_BK_LAUNCH(19) CECA_BK_LAUNCH(20)
       CECA_BK_LAUNCH(21)
@@ -634,7 +680,7 @@ ceca_status_t consensus_block(const float *X, const float *Y, float *Xo, float *
     }
 #undef CECA_BK_LAUNCH
   } else {
-#define CECA_BK_LAUNCH(CB) case CB: e = launch_block<CB, 8>(mx, my, a, g.threads, g.cmin, stream); break;
+#define CECA_BK_LAUNCH(CB) case CB: e = launch_block<CB, 8>(maps, a, g.threads, g.cmin, stream); break;
     switch (g.cb) {
       CECA_BK_LAUNCH(9) CECA_BK_LAUNCH(13) CECA_BK_LAUNCH(17) CECA_BK_LAUNCH(21) CECA_BK_LAUNCH(25)
       default: break;
