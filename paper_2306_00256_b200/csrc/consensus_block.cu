@@ -6,8 +6,9 @@
 // is two adjacent matrix columns of one block of agents: LPB threads side by side cover the 2 * LPB
 // columns of the tile, and each keeps I and J of a contiguous block of CB agents (rows i0 .. i0+CB-1)
 // of its two columns in registers, at static register positions.  LPB = 32 (a block is a warp, 64-column
-// tiles) serves n <= 256; LPB = 16 and 8 (32- and 16-column tiles, two and four blocks per warp) let
-// all rows of a tile fit on one SM up to n = 512 and n = 1152 (the paper's n = 1026).  Two ways of
+// tiles) serves n <= 200; LPB = 16 and 8 (32- and 16-column tiles, two and four blocks per warp) let
+// all rows of a tile fit on one SM, two CTAs at a time up to n = 400 and n = 800, and one up to n = 1152
+// (the paper's n = 1026).  Two ways of
 // cutting n rows into blocks, both with compile-time trip counts for every loop over a block:
 //   balanced (LPB >= 16): the first blocks hold CB agents, the others CB-1 (one predicated row);
 //   uniform (LPB = 8): every block holds CB agents except the last, which holds what is left; its
@@ -86,7 +87,6 @@ struct BlockArgs {
   int32_t boxes, box_rows;   // a tile lands as `boxes` TMA boxes of `box_rows` rows (boxes * box_rows >= n)
   uint32_t tile_bytes; // shared-memory footprint of one tile (a multiple of 128 that holds blocks * CB rows and all boxes)
   int32_t single_xch;  // one exchange tile instead of two (saves shared memory, costs a second barrier per round)
-  int32_t tma_out;     // results leave through the exchange tiles and TMA tensor stores instead of register stores
   int32_t wait_polls;
   uint32_t tx_bytes;   // bytes the landing barrier is armed for
   float outI, outJ;
@@ -257,12 +257,10 @@ __device__ __forceinline__ void dispatch_round(int sel, int s, int n, pk2 (&Ih)[
 template <int CB, int LPB, int MAXT>
 __global__ void __launch_bounds__(MAXT, 1)
 consensus_block_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_y,
-                       const __grid_constant__ CUtensorMap map_xo, const __grid_constant__ CUtensorMap map_yo,
                        const __grid_constant__ BlockArgs p) {
   constexpr int kTileCols = 2 * LPB;
   constexpr int RB = kTileCols * (int)sizeof(float);
   constexpr bool kBalanced = LPB >= 16;
-  constexpr bool kTmaOut = LPB < 32;   // the TMA-store form exists for the narrow tiles only (a launch parameter picks it)
   // received rows in flight per thread: eight, or four where the state leaves fewer than 36 other registers
   constexpr int kInFlight = 65536 / MAXT - 4 * CB >= 36 ? 8 : 4;
   extern __shared__ __align__(128) unsigned char smem_raw[];
@@ -318,11 +316,9 @@ consensus_block_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
       // that it cannot write into shared memory of a finished CTA) and give up without storing.
       if (threadIdx.x == 0) atomicExch(p.status, 1);
       mbar_wait_bounded(&bar, phase, (uint32_t)p.wait_polls);
-      if (kTmaOut && threadIdx.x == 0) tma_store_wait_read();   // an earlier tile's stores still read shared memory
       return;
     }
     phase ^= 1u;
-    bool staging_free = false;   // TMA-store form: the previous tile's stores have finished reading the exchange tiles
 
     pk2 Ih[CB], Jh[CB];
     {
@@ -371,12 +367,6 @@ consensus_block_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
         // the first round's neighbours) are done: the next tile may land while this one is finished
         issue_load(next_tile);
       }
-      if (kTmaOut && p.tma_out && rnd == 1) {
-        // the first publish of this tile: the previous tile's TMA stores must be done with the exchange tiles
-        if (threadIdx.x == 0) tma_store_wait_read();
-        __syncthreads();
-        staging_free = true;
-      }
       // The first round finds every row's payload in the landed tile and publishes nothing.
       q.publish = rnd > 0;
       const uint32_t buf_tile = rnd == 0 ? ((mode & kBkPayloadJ) ? y_tile : 0u) : ((rnd & 1) || p.single_xch ? 1u : 2u);
@@ -390,36 +380,8 @@ consensus_block_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
     }
 
     const int32_t col = tile * kTileCols + 2 * lane;
-    if (kTmaOut && p.tma_out) {
-      // Results go into the two exchange tiles (X+ into the first, Y+ into the second) and leave as TMA
-      // tensor stores, which clip at row n and column d.  The CTA does not wait for them: they drain
-      // while the next tile lands and runs its first round, which touches neither exchange tile.
-      if (!staging_free && threadIdx.x == 0) tma_store_wait_read();
-      __syncthreads();   // the last round's reads of the exchange tiles are done (and the old stores, see above)
-      const pk2 oI = pk_make(p.outI, p.outI), oJ = pk_make(p.outJ, p.outJ);
-      const uint32_t sx = sm_land_x + p.tile_bytes + own_off, sy = sx + p.tile_bytes;
-      static_for<CB>([&](auto J) {
-        constexpr int j = CECA_IDX(J);
-        if (!kBalanced || j < CB - 1 || q.full) sts64<j * RB>(sx, mul2(oI, Ih[j]));
-      });
-      if (p.has_y_out) {
-        static_for<CB>([&](auto J) {
-          constexpr int j = CECA_IDX(J);
-          if (!kBalanced || j < CB - 1 || q.full) sts64<j * RB>(sy, mul2(oJ, Jh[j]));
-        });
-      }
-      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic writes -> visible to the TMA unit
-      __syncthreads();
-      if (threadIdx.x == 0) {
-        for (int b = 0; b < p.boxes; ++b) {
-          const int row0 = b * p.box_rows;
-          tma_store_2d(&map_xo, tile * kTileCols, row0, smem_raw + p.tile_bytes + (size_t)row0 * RB);
-          if (p.has_y_out) tma_store_2d(&map_yo, tile * kTileCols, row0, smem_raw + 2 * (size_t)p.tile_bytes + (size_t)row0 * RB);
-        }
-        tma_store_commit();
-      }
-    } else if (LPB < 32 && (int)(threadIdx.x / LPB) >= p.blocks) {
-      // surplus threads (only where a block is narrower than a warp) shadow the last block and write nothing
+    // surplus threads (only where a block is narrower than a warp) shadow the last block and write nothing
+    if (LPB < 32 && (int)(threadIdx.x / LPB) >= p.blocks) {
     } else if (col + 1 < p.d) {
       const pk2 oI = pk_make(p.outI, p.outI), oJ = pk_make(p.outJ, p.outJ);
       float *dst = p.Xo + (int64_t)q.i0 * p.ld + col;
@@ -457,7 +419,6 @@ consensus_block_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
       if (threadIdx.x == 0) issue_load(next_tile);
     }
   }
-  if (kTmaOut && p.tma_out && threadIdx.x == 0) tma_store_wait_read();   // shared memory must outlive the stores' reads
 }
 
 // ---- host side ----------------------------------------------------------------------------------
@@ -465,31 +426,41 @@ consensus_block_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
 constexpr size_t kBkSmemLimit = 227 * 1024 - 1024;   // opt-in maximum per CTA minus the static part
 
 // Geometry by n: threads per block of agents (tile = 2 * LPB columns), number of blocks, agents per block.
-//   LPB = 32 (n <= 256): blocks are warps; as few and as large as the register file allows (25 agents
+//   LPB = 32 (n <= 200): blocks are warps; as few and as large as the register file allows (25 agents
 //     take 100 state registers), because a round whose shift reaches the block size exchanges every
 //     row through shared memory and there are about log2(blocks) such rounds; 1, 2 or a multiple of 4
 //     warps, so that the warps of a CTA, which move in lockstep from barrier to barrier, load the four
-//     schedulers of an SM evenly (5, 6, 7 or 9 warps measured 15-40 % slower than 4 or 8).
-//   LPB = 16 (n <= 512), LPB = 8 (n <= 1152): narrower tiles, so that all n rows of a tile (three
-//     tiles' worth: landed, two exchange tiles) still fit in shared memory, in at most 512 threads.
-//     LPB = 8 takes an odd CB from a short list (see the bank argument at the top).
+//     schedulers of an SM evenly (5, 6, 7 or 9 warps measured 15-40 % slower than 4 or 8).  Twelve warps of
+//     22 agents (n = 201-256) leave one CTA per SM and lose 15-20 % to 32-column tiles with two.
+//   LPB = 16 (n <= 400), LPB = 8 (n <= 1152): narrower tiles, so that all n rows of a tile (three
+//     tiles' worth: landed, two exchange tiles) still fit in shared memory.  Two candidates each, and
+//     the launch takes the one that puts more CTAs on an SM (the compact one on a tie):
+//       `kBkCompact`: at most 256 threads (16 resp. 32 blocks of up to 25 agents), which at 128
+//         registers fits two CTAs per SM where shared memory allows it too -- measured 20-35 % faster
+//         than one CTA per SM (n = 350-400, 600-800), even where the 128-register form spills a little;
+//       `kBkPlain`: LPB = 16: blocks of 20-23 agents, sizes whose 128-register form does not spill;
+//         LPB = 8: up to 512 threads of small blocks, the best of the one-CTA-per-SM shapes measured.
+//     LPB = 8 needs an odd CB (see the bank argument at the top).
 struct BlockGeom {
   int lpb, cb, blocks, threads;
   int nfull;   // see BlockArgs
   int cmin;    // size of the smallest block that a partial round's source rows may lie in
 };
 constexpr int kBkMaxRows = 1152;
-static bool block_geometry(int n, int warps_override, BlockGeom *g) {
+constexpr int kBkPlain = 0, kBkCompact = 1;
+static bool block_geometry(int n, int warps_override, int kind, BlockGeom *g) {
   if (n < 2 || n > kBkMaxRows) return false;
-  if (n <= 512) {
+  if (n <= 400) {
     int blocks;
-    if (n <= 256) {
+    if (n <= 200) {
+      if (kind != kBkPlain) return false;
       g->lpb = 32;
-      blocks = n <= 25 ? 1 : n <= 50 ? 2 : n <= 100 ? 4 : n <= 200 ? 8 : 12;
+      blocks = n <= 25 ? 1 : n <= 50 ? 2 : n <= 100 ? 4 : 8;
       if (warps_override > 0) blocks = warps_override;
     } else {
       g->lpb = 16;
-      blocks = n <= 336 ? 16 : n <= 504 ? 24 : 32;
+      if (kind == kBkCompact) blocks = 16;
+      else blocks = ((n + 22) / 23 + 1) / 2 * 2;   // an even number of blocks of at most 23 agents: whole warps
     }
     if (blocks > n) blocks = n;
     g->blocks = blocks;
@@ -498,11 +469,17 @@ static bool block_geometry(int n, int warps_override, BlockGeom *g) {
     g->cmin = g->nfull == blocks ? g->cb : g->cb - 1;
   } else {
     g->lpb = 8;
-    static const int kSizes[] = {9, 13, 17, 21, 25};
-    g->cb = 0;
-    for (int cb : kSizes)
-      if ((n + cb - 1) / cb <= 512 / g->lpb) { g->cb = cb; break; }
-    if (!g->cb) return false;
+    if (kind == kBkCompact) {
+      g->cb = 25;   // few, roomy threads: blocks of 17-23 agents in up to 256 threads measured 15-30 % slower
+      if ((n + 24) / 25 > 32) return false;   // more than 256 threads: one CTA per SM anyway
+    } else {
+      // one CTA per SM: many threads, the smallest size that fits in 512 of them
+      static const int kSizes[] = {9, 13, 17, 21, 25};
+      g->cb = 0;
+      for (int cb : kSizes)
+        if ((n + cb - 1) / cb <= 512 / g->lpb) { g->cb = cb; break; }
+      if (!g->cb) return false;
+    }
     g->blocks = (n + g->cb - 1) / g->cb;
     g->nfull = n / g->cb;
     g->cmin = g->cb;   // the sources of a partial round lie in full blocks, or are all published (last block)
@@ -530,14 +507,16 @@ static BlockTile block_tile(int n, const BlockGeom &g) {
 
 // y_in: the first round reads Y, which takes one more shared-memory tile (at least two are needed without it).
 bool consensus_block_supports(int32_t n, ceca_variant_t variant, int32_t rounds, bool y_in) {
-  BlockGeom g;
-  if (variant != CECA_2P || rounds < 1 || rounds > kBkMaxRounds || !block_geometry(n, 0, &g)) return false;
-  return (size_t)(y_in ? 3 : 2) * block_tile(n, g).tile_bytes <= kBkSmemLimit;
+  if (variant != CECA_2P || rounds < 1 || rounds > kBkMaxRounds) return false;
+  for (int kind = 0; kind < 2; ++kind) {
+    BlockGeom g;
+    if (block_geometry(n, 0, kind, &g) && (size_t)(y_in ? 3 : 2) * block_tile(n, g).tile_bytes <= kBkSmemLimit) return true;
+  }
+  return false;
 }
 
 // Register budgets by block size (the state takes 4 * CB registers): a roomy one, and a lean one that
 // still compiles without spilling to speak of.  65536 / kMaxThreads registers per thread.
-constexpr int kBkTmaOutMaxCtas = 2;
 template <int CB> struct BlockRegs {
   static constexpr int kRoomy = CB >= 15 ? 384 : CB >= 11 ? 640 : CB >= 7 ? 768 : 1024;
   static constexpr int kLean = CB >= 15 ? 512 : CB >= 11 ? 768 : 1024;
@@ -561,12 +540,14 @@ static cudaError_t launch_block_regs(const CUtensorMap *maps, const BlockArgs &a
   // persistent CTAs: as many as fit on the device at once, not more than there are tiles
   const int64_t resident = (int64_t)sms * per_sm;
   const int grid = (int)(a.tiles < resident ? a.tiles : resident);
-  consensus_block_kernel<CB, LPB, MAXT><<<grid, threads, smem, stream>>>(maps[0], maps[1], maps[2], maps[3], a);
+  consensus_block_kernel<CB, LPB, MAXT><<<grid, threads, smem, stream>>>(maps[0], maps[1], a);
   return cudaGetLastError();
 }
 
+// launch == false: only reports in *ctas_per_sm how many CTAs of the best launch shape share an SM.
 template <int CB, int LPB>
-static cudaError_t launch_block(const CUtensorMap *maps, BlockArgs &a, int threads, int cmin, cudaStream_t stream) {
+static cudaError_t launch_block(const CUtensorMap *maps, BlockArgs &a, int threads, int cmin, bool launch,
+                                int *ctas_per_sm, cudaStream_t stream) {
   for (int t = 0; t < a.rounds; ++t) {
     BlockRound &r = a.rd[t];
     const int pay = (r.mode & kBkPayloadJ) ? 1 : 0;
@@ -592,22 +573,73 @@ static cudaError_t launch_block(const CUtensorMap *maps, BlockArgs &a, int threa
     if (roomy > best) { best = roomy; best_single = single; best_lean = 0; }
     if (lean > best) { best = lean; best_single = single; best_lean = 1; }
   }
+  *ctas_per_sm = best;
   if (best < 1) return cudaErrorInvalidConfiguration;
+  if (!launch) return cudaSuccess;
   a.single_xch = best_single;
-  // Narrow tiles with both exchange tiles and at most kBkTmaOutMaxCtas CTAs per SM: register stores would hold
-  // the whole CTA (and with it the SM) until the memory system has taken them; TMA stores from the
-  // exchange tiles let the next tile start meanwhile.
-  a.tma_out = (LPB < 32 && !best_single && best <= kBkTmaOutMaxCtas) ? 1 : 0;
   const size_t smem = ((a.has_y_in ? 2 : 1) + (best_single ? 1 : 2)) * tile_bytes;
   int per_sm = 0;
   if (best_lean) return launch_block_regs<CB, LPB, kLean>(maps, a, threads, smem, &per_sm, true, stream);
   return launch_block_regs<CB, LPB, kRoomy>(maps, a, threads, smem, &per_sm, true, stream);
 }
 
+// Fills the geometry-dependent launch arguments for candidate `kind` and either launches it or only
+// reports its CTAs per SM.  CECA_ERR_UNSUPPORTED: this candidate does not exist for n or does not fit.
+static ceca_status_t block_dispatch(const float *X, const float *Y, float *Xo, float *Yo, int32_t n, int64_t d, int64_t ld,
+                                    BlockArgs &a, int kind, int warps_override, uint32_t tx_extra, bool launch,
+                                    int *ctas_per_sm, cudaStream_t stream) {
+  BlockGeom g;
+  if (!block_geometry(n, warps_override, kind, &g)) return CECA_ERR_UNSUPPORTED;
+  const BlockTile t = block_tile(n, g);
+  if ((size_t)(a.has_y_in ? 3 : 2) * t.tile_bytes > kBkSmemLimit) return CECA_ERR_UNSUPPORTED;
+  const int tile_cols = 2 * g.lpb;
+  a.blocks = g.blocks; a.nfull = g.nfull; a.boxes = t.boxes; a.box_rows = t.box_rows; a.tile_bytes = (uint32_t)t.tile_bytes;
+  a.tiles = (int32_t)((d + tile_cols - 1) / tile_cols);
+  // a box counts in full towards the barrier, rows and columns outside the matrix included
+  a.tx_bytes = (uint32_t)t.boxes * t.box_rows * tile_cols * sizeof(float) * (a.has_y_in ? 2u : 1u) + tx_extra;
+
+  CUtensorMap maps[2];   // X in, Y in (X again when Y is not read)
+  if (launch) {
+    if (!tensor_map_2d(&maps[0], X, n, d, ld, tile_cols, t.box_rows)) return CECA_ERR_CUDA;
+    if (!tensor_map_2d(&maps[1], a.has_y_in ? Y : X, n, d, ld, tile_cols, t.box_rows)) return CECA_ERR_CUDA;
+  }
+
+  cudaError_t e = cudaErrorInvalidConfiguration;
+#define CECA_BK_LAUNCH(CB) case CB: e = launch_block<CB, kLpb>(maps, a, g.threads, g.cmin, launch, ctas_per_sm, stream); break;
+  if (g.lpb == 32) {
+    constexpr int kLpb = 32;
+    switch (g.cb) {
+      CECA_BK_LAUNCH(1) CECA_BK_LAUNCH(2) CECA_BK_LAUNCH(3) CECA_BK_LAUNCH(4) CECA_BK_LAUNCH(5) CECA_BK_LAUNCH(6)
+      CECA_BK_LAUNCH(7) CECA_BK_LAUNCH(8) CECA_BK_LAUNCH(9) CECA_BK_LAUNCH(10) CECA_BK_LAUNCH(11) CECA_BK_LAUNCH(12)
+      CECA_BK_LAUNCH(13) CECA_BK_LAUNCH(14) CECA_BK_LAUNCH(15) CECA_BK_LAUNCH(16) CECA_BK_LAUNCH(17) CECA_BK_LAUNCH(18)
+      CECA_BK_LAUNCH(19) CECA_BK_LAUNCH(20) CECA_BK_LAUNCH(21) CECA_BK_LAUNCH(22) CECA_BK_LAUNCH(23) CECA_BK_LAUNCH(24)
+      CECA_BK_LAUNCH(25)
+      default: break;
+    }
+  } else if (g.lpb == 16) {
+    constexpr int kLpb = 16;
+    switch (g.cb) {   // n = 201 .. 400: 16 blocks of 13 to 25 agents, or 10 to 18 blocks of 20 to 23
+      CECA_BK_LAUNCH(13) CECA_BK_LAUNCH(14) CECA_BK_LAUNCH(15) CECA_BK_LAUNCH(16) CECA_BK_LAUNCH(17) CECA_BK_LAUNCH(18)
+      CECA_BK_LAUNCH(19) CECA_BK_LAUNCH(20) CECA_BK_LAUNCH(21) CECA_BK_LAUNCH(22) CECA_BK_LAUNCH(23) CECA_BK_LAUNCH(24)
+      CECA_BK_LAUNCH(25)
+      default: break;
+    }
+  } else {
+    constexpr int kLpb = 8;
+    switch (g.cb) {   // n = 513 .. 1152: odd sizes
+      CECA_BK_LAUNCH(9) CECA_BK_LAUNCH(13) CECA_BK_LAUNCH(17) CECA_BK_LAUNCH(21) CECA_BK_LAUNCH(25)
+      default: break;
+    }
+  }
+#undef CECA_BK_LAUNCH
+  if (e == cudaErrorInvalidConfiguration) return CECA_ERR_UNSUPPORTED;
+  return e == cudaSuccess ? CECA_OK : CECA_ERR_CUDA;
+}
+
 // Arguments are assumed validated by the caller (shapes, aliasing, 16-byte alignment of X / Y and
 // ld % 4 == 0, d and ld within 32 bits, Y present when the first round reads it, status word).
 // The caller has checked consensus_block_supports.  `warps_override` > 0 forces the number of
-// blocks for n <= 256 (used to measure the alternatives).
+// blocks for n <= 200 (used to measure the alternatives).
 ceca_status_t consensus_block(const float *X, const float *Y, float *Xo, float *Yo, int32_t n, int64_t d,
                               int64_t ld, int64_t k0, int32_t rounds, int32_t *status, int32_t wait_polls,
                               uint32_t tx_extra, int warps_override, cudaStream_t stream) {
@@ -644,51 +676,17 @@ ceca_status_t consensus_block(const float *X, const float *Y, float *Xo, float *
   a.has_y_in = (Y != nullptr && first_needs_y) ? 1 : 0;
   if (!consensus_block_supports(n, CECA_2P, rounds, a.has_y_in != 0)) return CECA_ERR_UNSUPPORTED;
 
-  BlockGeom g;
-  if (!block_geometry(n, warps_override, &g)) return CECA_ERR_UNSUPPORTED;
-  const BlockTile t = block_tile(n, g);
-  const int tile_cols = 2 * g.lpb;
-  a.blocks = g.blocks; a.nfull = g.nfull; a.boxes = t.boxes; a.box_rows = t.box_rows; a.tile_bytes = (uint32_t)t.tile_bytes;
-  a.tiles = (int32_t)((d + tile_cols - 1) / tile_cols);
-  // a box counts in full towards the barrier, rows and columns outside the matrix included
-  a.tx_bytes = (uint32_t)t.boxes * t.box_rows * tile_cols * sizeof(float) * (a.has_y_in ? 2u : 1u) + tx_extra;
-
-  CUtensorMap maps[4];   // X in, Y in, X out, Y out (unused ones alias a used one)
-  if (!tensor_map_2d(&maps[0], X, n, d, ld, tile_cols, t.box_rows)) return CECA_ERR_CUDA;
-  if (!tensor_map_2d(&maps[1], a.has_y_in ? Y : X, n, d, ld, tile_cols, t.box_rows)) return CECA_ERR_CUDA;
-  if (!tensor_map_2d(&maps[2], Xo, n, d, ld, tile_cols, t.box_rows)) return CECA_ERR_CUDA;
-  if (!tensor_map_2d(&maps[3], Yo ? Yo : Xo, n, d, ld, tile_cols, t.box_rows)) return CECA_ERR_CUDA;
-
-  cudaError_t e = cudaErrorInvalidConfiguration;
-  if (g.lpb == 32) {
-    switch (g.cb) {
-#define CECA_BK_LAUNCH(CB) case CB: e = launch_block<CB, 32>(maps, a, g.threads, g.cmin, stream); break;
-      CECA_BK_LAUNCH(1) CECA_BK_LAUNCH(2) CECA_BK_LAUNCH(3) CECA_BK_LAUNCH(4) CECA_BK_LAUNCH(5) CECA_BK_LAUNCH(6)
-      CECA_BK_LAUNCH(7) CECA_BK_LAUNCH(8) CECA_BK_LAUNCH(9) CECA_BK_LAUNCH(10) CECA_BK_LAUNCH(11) CECA_BK_LAUNCH(12)
-      CECA_BK_LAUNCH(13) CECA_BK_LAUNCH(14) CECA_BK_LAUNCH(15) CECA_BK_LAUNCH(16) CECA_BK_LAUNCH(17) CECA_BK_LAUNCH(18)
-      CECA_BK_LAUNCH(19) CECA_BK_LAUNCH(20) CECA_BK_LAUNCH(21) CECA_BK_LAUNCH(22) CECA_BK_LAUNCH(23) CECA_BK_LAUNCH(24)
-      CECA_BK_LAUNCH(25)
-#undef CECA_BK_LAUNCH
-      default: break;
-    }
-  } else if (g.lpb == 16) {
-#define CECA_BK_LAUNCH(CB) case CB: e = launch_block<CB, 16>(maps, a, g.threads, g.cmin, stream); break;
-    switch (g.cb) {   // n = 257 .. 512 in 16, 24 or 32 blocks: 15 to 21 agents per block
-      CECA_BK_LAUNCH(15) CECA_BK_LAUNCH(16) CECA_BK_LAUNCH(17) CECA_BK_LAUNCH(18) CECA_BK_LAUNCH(19) CECA_BK_LAUNCH(20)
-      CECA_BK_LAUNCH(21)
-      default: break;
-    }
-#undef CECA_BK_LAUNCH
-  } else {
-#define CECA_BK_LAUNCH(CB) case CB: e = launch_block<CB, 8>(maps, a, g.threads, g.cmin, stream); break;
-    switch (g.cb) {
-      CECA_BK_LAUNCH(9) CECA_BK_LAUNCH(13) CECA_BK_LAUNCH(17) CECA_BK_LAUNCH(21) CECA_BK_LAUNCH(25)
-      default: break;
-    }
-#undef CECA_BK_LAUNCH
+  // The candidate geometries are asked how many CTAs they put on an SM; the first of the best is launched.
+  int best_kind = -1, best_ctas = 0;
+  for (int kind = 1; kind >= 0; --kind) {   // the compact candidate first: it wins ties
+    int ctas = 0;
+    const ceca_status_t st = block_dispatch(X, Y, Xo, Yo, n, d, ld, a, kind, warps_override, tx_extra, false, &ctas, stream);
+    if (st == CECA_OK && ctas > best_ctas) { best_ctas = ctas; best_kind = kind; }
+    else if (st != CECA_OK && st != CECA_ERR_UNSUPPORTED) return st;
   }
-  if (e == cudaErrorInvalidConfiguration) return CECA_ERR_UNSUPPORTED;
-  return e == cudaSuccess ? CECA_OK : CECA_ERR_CUDA;
+  if (best_kind < 0) return CECA_ERR_UNSUPPORTED;
+  int ctas = 0;
+  return block_dispatch(X, Y, Xo, Yo, n, d, ld, a, best_kind, warps_override, tx_extra, true, &ctas, stream);
 }
 
 }  // namespace ceca

@@ -55,10 +55,6 @@ __device__ __forceinline__ void tma_store_2d(const CUtensorMap *map, int32_t x, 
                ::"l"(map), "r"(x), "r"(y), "r"(smem_u32(src))
                : "memory");
 }
-__device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
-// Waits until every committed tensor store of this thread has finished READING shared memory (the
-// global writes may still be under way): after it the source tiles may be overwritten.
-__device__ __forceinline__ void tma_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
 #endif  // __CUDACC__
 
 // The tensor map of an n x d fp32 matrix with row pitch ld (elements), boxed as box_rows rows x

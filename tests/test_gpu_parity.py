@@ -294,7 +294,7 @@ def _fused_kernels(n, variant=ceca.CECA_2P):
 
 
 @pytest.mark.parametrize("fused", [ceca.UNFUSED, ceca.FUSED_SMEM, ceca.FUSED_TMEM, ceca.FUSED_BLOCK])
-@pytest.mark.parametrize("n", [2, 3, 4, 5, 6, 7, 8, 9, 16, 17, 24, 31, 33, 63, 65, 97, 100, 127, 128, 129, 130, 200, 255, 256])
+@pytest.mark.parametrize("n", [2, 3, 4, 5, 6, 7, 8, 9, 16, 17, 24, 31, 33, 63, 65, 97, 100, 127, 128, 129, 130, 200, 201, 208, 209, 255, 256])
 @pytest.mark.parametrize("d", [32, 1000, 4100])
 def test_consensus_matches_oracle_and_reaches_the_mean(fused, n, d):
     if fused == ceca.FUSED_TMEM and n > 128:
@@ -333,7 +333,7 @@ def test_consensus_matches_oracle_and_reaches_the_mean(fused, n, d):
 
 
 @pytest.mark.parametrize("fused", [ceca.FUSED_AUTO, ceca.FUSED_SMEM, ceca.FUSED_BLOCK])
-@pytest.mark.parametrize("n", [257, 258, 300, 511, 512, 513, 514, 1026, 1087, 1088, 1089, 1152, 1153, 1300, 2047, 2048])
+@pytest.mark.parametrize("n", [257, 258, 300, 367, 368, 369, 400, 401, 512, 513, 600, 800, 801, 1026, 1089, 1151, 1152, 1153, 1300, 2047, 2048])
 @pytest.mark.parametrize("d", [8, 1000, 4100])
 def test_fused_consensus_above_256_agents(fused, n, d):
     """Tiles taller than one TMA box (32-, 16- or 8-column tiles made of several boxes): tau rounds, extra rounds,
