@@ -98,10 +98,10 @@ NCU_TRAFFIC = {
     "logreg_grad": (2.1034e9, "dram_traffic__step_consensus_gradient.md", "logreg.cu", "b3cedf2f4e6b"),
     "logreg_grad_d32768": (2.1357e9, "dram_traffic__step_consensus_gradient.md", "logreg.cu", "b3cedf2f4e6b"),
     # register-block kernel: captured at d = 2^19 (0.5522 GB per launch) and doubled for d = 2^20 (traffic is per tile)
-    "consensus_fused_small": (0.5522e9, "consensus_block_kernel__n97_n258_n1026__ncu_full.md", "consensus_block.cu", "cab05557c0cc"),
-    "consensus_fused": (1.1044e9, "consensus_block_kernel__n97_n258_n1026__ncu_full.md", "consensus_block.cu", "cab05557c0cc"),
-    "consensus_fused_258": (1.5641e9, "consensus_block_kernel__n97_n258_n1026__ncu_full.md", "consensus_block.cu", "cab05557c0cc"),
-    "consensus_fused_1026": (3.1769e9, "consensus_block_kernel__n97_n258_n1026__ncu_full.md", "consensus_block.cu", "cab05557c0cc"),
+    "consensus_fused_small": (0.5522e9, "consensus_block_kernel__n97_n258_n1026__ncu_full.md", "consensus_block.cu", "45b50a63710f"),
+    "consensus_fused": (1.1044e9, "consensus_block_kernel__n97_n258_n1026__ncu_full.md", "consensus_block.cu", "45b50a63710f"),
+    "consensus_fused_258": (1.5641e9, "consensus_block_kernel__n97_n258_n1026__ncu_full.md", "consensus_block.cu", "45b50a63710f"),
+    "consensus_fused_1026": (3.1769e9, "consensus_block_kernel__n97_n258_n1026__ncu_full.md", "consensus_block.cu", "45b50a63710f"),
 }
 
 

@@ -6,7 +6,7 @@
 // is two adjacent matrix columns of one block of agents: LPB threads side by side cover the 2 * LPB
 // columns of the tile, and each keeps I and J of a contiguous block of CB agents (rows i0 .. i0+CB-1)
 // of its two columns in registers, at static register positions.  LPB = 32 (a block is a warp, 64-column
-// tiles) serves n <= 200; LPB = 16 and 8 (32- and 16-column tiles, two and four blocks per warp) let
+// tiles) serves n <= 150; LPB = 16 and 8 (32- and 16-column tiles, two and four blocks per warp) let
 // all rows of a tile fit on one SM, two CTAs at a time up to n = 400 and n = 800, and one up to n = 1152
 // (the paper's n = 1026).  Two ways of
 // cutting n rows into blocks, both with compile-time trip counts for every loop over a block:
@@ -426,16 +426,17 @@ consensus_block_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
 constexpr size_t kBkSmemLimit = 227 * 1024 - 1024;   // opt-in maximum per CTA minus the static part
 
 // Geometry by n: threads per block of agents (tile = 2 * LPB columns), number of blocks, agents per block.
-//   LPB = 32 (n <= 200): blocks are warps; as few and as large as the register file allows (25 agents
+//   LPB = 32 (n <= 150): blocks are warps; as few and as large as the register file allows (25 agents
 //     take 100 state registers), because a round whose shift reaches the block size exchanges every
 //     row through shared memory and there are about log2(blocks) such rounds; 1, 2 or a multiple of 4
 //     warps, so that the warps of a CTA, which move in lockstep from barrier to barrier, load the four
 //     schedulers of an SM evenly (5, 6, 7 or 9 warps measured 15-40 % slower than 4 or 8).  Twelve warps of
-//     22 agents (n = 201-256) leave one CTA per SM and lose 15-20 % to 32-column tiles with two.
+//     22 agents (n = 201-256) leave one CTA per SM and lose 15-20 % to 32-column tiles with two; from
+//     n = 150 on eight half-warp blocks (128 threads, more CTAs per SM) are 5-9 % faster than eight warps.
 //   LPB = 16 (n <= 400), LPB = 8 (n <= 1152): narrower tiles, so that all n rows of a tile (three
 //     tiles' worth: landed, two exchange tiles) still fit in shared memory.  Two candidates each, and
 //     the launch takes the one that puts more CTAs on an SM (the compact one on a tie):
-//       `kBkCompact`: at most 256 threads (16 resp. 32 blocks of up to 25 agents), which at 128
+//       `kBkCompact`: at most 256 threads (8 or 16 resp. 32 blocks of up to 25 agents), which at 128
 //         registers fits two CTAs per SM where shared memory allows it too -- measured 20-35 % faster
 //         than one CTA per SM (n = 350-400, 600-800), even where the 128-register form spills a little;
 //       `kBkPlain`: LPB = 16: blocks of 20-23 agents, sizes whose 128-register form does not spill;
@@ -452,14 +453,14 @@ static bool block_geometry(int n, int warps_override, int kind, BlockGeom *g) {
   if (n < 2 || n > kBkMaxRows) return false;
   if (n <= 400) {
     int blocks;
-    if (n <= 200) {
+    if (n <= 150) {
       if (kind != kBkPlain) return false;
       g->lpb = 32;
       blocks = n <= 25 ? 1 : n <= 50 ? 2 : n <= 100 ? 4 : 8;
       if (warps_override > 0) blocks = warps_override;
     } else {
       g->lpb = 16;
-      if (kind == kBkCompact) blocks = 16;
+      if (kind == kBkCompact) blocks = n <= 200 ? 8 : 16;
       else blocks = ((n + 22) / 23 + 1) / 2 * 2;   // an even number of blocks of at most 23 agents: whole warps
     }
     if (blocks > n) blocks = n;
@@ -618,7 +619,7 @@ static ceca_status_t block_dispatch(const float *X, const float *Y, float *Xo, f
     }
   } else if (g.lpb == 16) {
     constexpr int kLpb = 16;
-    switch (g.cb) {   // n = 201 .. 400: 16 blocks of 13 to 25 agents, or 10 to 18 blocks of 20 to 23
+    switch (g.cb) {   // n = 151 .. 400: 8 or 16 blocks of 13 to 25 agents, or 8 to 18 blocks of 19 to 23
       CECA_BK_LAUNCH(13) CECA_BK_LAUNCH(14) CECA_BK_LAUNCH(15) CECA_BK_LAUNCH(16) CECA_BK_LAUNCH(17) CECA_BK_LAUNCH(18)
       CECA_BK_LAUNCH(19) CECA_BK_LAUNCH(20) CECA_BK_LAUNCH(21) CECA_BK_LAUNCH(22) CECA_BK_LAUNCH(23) CECA_BK_LAUNCH(24)
       CECA_BK_LAUNCH(25)
@@ -639,7 +640,7 @@ static ceca_status_t block_dispatch(const float *X, const float *Y, float *Xo, f
 // Arguments are assumed validated by the caller (shapes, aliasing, 16-byte alignment of X / Y and
 // ld % 4 == 0, d and ld within 32 bits, Y present when the first round reads it, status word).
 // The caller has checked consensus_block_supports.  `warps_override` > 0 forces the number of
-// blocks for n <= 200 (used to measure the alternatives).
+// blocks for n <= 150 (used to measure the alternatives).
 ceca_status_t consensus_block(const float *X, const float *Y, float *Xo, float *Yo, int32_t n, int64_t d,
                               int64_t ld, int64_t k0, int32_t rounds, int32_t *status, int32_t wait_polls,
                               uint32_t tx_extra, int warps_override, cudaStream_t stream) {

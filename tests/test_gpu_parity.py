@@ -294,7 +294,7 @@ def _fused_kernels(n, variant=ceca.CECA_2P):
 
 
 @pytest.mark.parametrize("fused", [ceca.UNFUSED, ceca.FUSED_SMEM, ceca.FUSED_TMEM, ceca.FUSED_BLOCK])
-@pytest.mark.parametrize("n", [2, 3, 4, 5, 6, 7, 8, 9, 16, 17, 24, 31, 33, 63, 65, 97, 100, 127, 128, 129, 130, 200, 201, 208, 209, 255, 256])
+@pytest.mark.parametrize("n", [2, 3, 4, 5, 6, 7, 8, 9, 16, 17, 24, 31, 33, 63, 65, 97, 100, 127, 128, 129, 130, 150, 151, 161, 200, 201, 208, 209, 255, 256])
 @pytest.mark.parametrize("d", [32, 1000, 4100])
 def test_consensus_matches_oracle_and_reaches_the_mean(fused, n, d):
     if fused == ceca.FUSED_TMEM and n > 128:
