@@ -66,7 +66,7 @@ WORKLOADS = {
     "consensus_fused_1026_smem": dict(kind="consensus", n=1026, d=1 << 18, variant=2, fused=2),
     "consensus_rounds_1026": dict(kind="consensus", n=1026, d=1 << 18, variant=2, fused=0),
     "logreg_grad": dict(kind="logreg", n=63, m=2000, d=4096, variant=2, gamma=0.01),
-    # wider models at the same 2 GB of samples: eight float4 per thread (d = 8192), clusters of 8 CTAs of 4096 columns (d = 32768)
+    # wider models at the same 2 GB of samples: 512 threads per CTA (d = 8192), clusters of 4 and 8 CTAs of 4096 columns
     "logreg_grad_d8192": dict(kind="logreg", n=32, m=2000, d=8192, variant=2, gamma=0.01),
     "logreg_grad_d16384": dict(kind="logreg", n=16, m=2000, d=16384, variant=2, gamma=0.01),
     "logreg_grad_d32768": dict(kind="logreg", n=8, m=2000, d=32768, variant=2, gamma=0.01),
@@ -95,8 +95,8 @@ NCU_TRAFFIC = {
     # seven launches of a cycle: round 0 moves 1.168 GB, the six others 1.565 GB each
     "consensus_rounds": (10.558e9, "dram_traffic__step_consensus_gradient.md", "step.cu", "b16a43e291d9"),
     # fused kernel 2.0735 GB + fixed-order reduce 0.0299 GB
-    "logreg_grad": (2.1034e9, "dram_traffic__step_consensus_gradient.md", "logreg.cu", "b3cedf2f4e6b"),
-    "logreg_grad_d32768": (2.1357e9, "dram_traffic__step_consensus_gradient.md", "logreg.cu", "b3cedf2f4e6b"),
+    "logreg_grad": (2.1034e9, "dram_traffic__step_consensus_gradient.md", "logreg.cu", "1bf7d97691f2"),
+    "logreg_grad_d32768": (2.1357e9, "dram_traffic__step_consensus_gradient.md", "logreg.cu", "1bf7d97691f2"),
     # register-block kernel: captured at d = 2^19 (0.5522 GB per launch) and doubled for d = 2^20 (traffic is per tile)
     "consensus_fused_small": (0.5522e9, "consensus_block_kernel__n97_n258_n1026__ncu_full.md", "consensus_block.cu", "45b50a63710f"),
     "consensus_fused": (1.1044e9, "consensus_block_kernel__n97_n258_n1026__ncu_full.md", "consensus_block.cu", "45b50a63710f"),

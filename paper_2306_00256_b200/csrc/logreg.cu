@@ -33,17 +33,15 @@
 
 namespace ceca {
 
-constexpr int kLrThreads = 256;
-constexpr int kLrWarps = kLrThreads / 32;
-constexpr int kLrMaxVpt = 8;         // float4 column groups per thread -> 256*4*8 = 8192 columns per CTA
+constexpr int kLrThreads = 256;      // threads per CTA; 512 for chunks wider than 4096 columns
+constexpr int kLrMaxVpt = 4;         // float4 column groups per thread -> 512*4*4 = 8192 columns per CTA
 constexpr int kLrMaxCluster = 8;     // CTAs (column chunks) per cluster: the portable maximum
-constexpr int kLrChunkCols = kLrThreads * 4 * kLrMaxVpt;
+constexpr int kLrChunkCols = 2 * kLrThreads * 4 * kLrMaxVpt;
 constexpr int kLrHalfChunkCols = kLrChunkCols / 2;   // four float4 per thread: two CTAs per SM, four rows in flight
 constexpr int kLrTargetCtas = 148 * 12;
 
-// Sample rows in flight per thread: four, or two where the thread's slice is so wide (eight float4
-// per row) that four rows of it would not fit in registers beside z and the gradient.
-template <int VPT> struct LrSamples { static constexpr int value = VPT >= 8 ? 2 : 4; };
+// Sample rows in flight per thread.
+template <int VPT> struct LrSamples { static constexpr int value = 4; };
 // NS inner products travel as one vector (one shared-memory access).
 template <int NS> struct LrDots;
 template <> struct LrDots<4> { using type = float4; };
@@ -56,8 +54,8 @@ __device__ __forceinline__ void dots_unpack(float4 v, float (&d)[4]) { d[0] = v.
 __device__ __forceinline__ void dots_unpack(float2 v, float (&d)[2]) { d[0] = v.x; d[1] = v.y; }
 
 // Column chunks (CTAs per cluster) for d columns.  One CTA while its registers hold the row
-// (d <= 8192: a cluster barrier per batch of rows costs more than the narrower slices win, 0.74
-// against 0.66 of the copy rate at d = 8192); beyond that chunks of 4096 columns (two CTAs per SM,
+// (d <= 8192: a cluster barrier per batch of rows costs more than it wins, 0.66 of the copy rate
+// for two CTAs of 4096 columns against 0.78 and more for one CTA at d = 8192); beyond that chunks of 4096 columns (two CTAs per SM,
 // four rows in flight) while a cluster of eight covers the row, chunks of up to 8192 columns above.
 static inline int32_t logreg_chunks(int64_t d) {
   if (d <= kLrChunkCols) return 1;
@@ -97,14 +95,17 @@ __device__ __forceinline__ float dot4(float4 a, float4 b) {
   return fmaf(a.x, b.x, fmaf(a.y, b.y, fmaf(a.z, b.z, a.w * b.w)));
 }
 
-// VPT float4 column groups per thread.  CLUSTER: launched as clusters of p.chunks CTAs along x; the
-// CTA of rank r takes the column groups [r * chunk4, (r + 1) * chunk4).
-template <int VPT, int LOSS, bool CLUSTER>
-__global__ void __launch_bounds__(kLrThreads, VPT == 1 ? 4 : VPT == 2 ? 3 : VPT == 4 ? 2 : 1)
+// T threads, VPT float4 column groups per thread (a chunk of up to T * VPT * 4 columns; 4096 < columns
+// <= 8192 take 512 threads of four groups rather than 256 of eight: the same registers per thread and
+// warps per SM as two CTAs of the 4096-column shape).  CLUSTER: launched as clusters of p.chunks CTAs
+// along x; the CTA of rank r takes the column groups [r * chunk4, (r + 1) * chunk4).
+template <int VPT, int LOSS, bool CLUSTER, int T>
+__global__ void __launch_bounds__(T, T > 256 ? 1 : VPT == 1 ? 4 : VPT == 2 ? 3 : 2)
 logreg_fused_kernel(const LogregArgs p) {
+  constexpr int kWarps = T / 32;
   constexpr int NS = LrSamples<VPT>::value;
   using Dots = typename LrDots<NS>::type;
-  __shared__ Dots red[2][kLrWarps];
+  __shared__ Dots red[2][kWarps];
   __shared__ Dots share[2][kLrMaxCluster];   // the inner-product shares of the cluster's CTAs
   namespace cg = cooperative_groups;
   const int rank = CLUSTER ? (int)cg::this_cluster().block_rank() : 0;
@@ -121,7 +122,7 @@ logreg_fused_kernel(const LogregArgs p) {
   bool valid[VPT];
 #pragma unroll
   for (int j = 0; j < VPT; ++j) {
-    const int64_t cgj = cg0 + threadIdx.x + (int64_t)j * kLrThreads;
+    const int64_t cgj = cg0 + threadIdx.x + (int64_t)j * T;
     valid[j] = cgj < cg_end;
     z[j] = valid[j] ? *reinterpret_cast<const float4 *>(p.Z + (int64_t)i * p.ld + cgj * 4)
                     : make_float4(0.f, 0.f, 0.f, 0.f);
@@ -142,7 +143,7 @@ logreg_fused_kernel(const LogregArgs p) {
       const float *row = a_agent + (int64_t)(s + jj) * p.d;
 #pragma unroll
       for (int j = 0; j < VPT; ++j) {
-        const int64_t cgl = threadIdx.x + (int64_t)j * kLrThreads;   // column group inside the chunk
+        const int64_t cgl = threadIdx.x + (int64_t)j * T;   // column group inside the chunk
         a[jj][j] = (live && valid[j]) ? __ldcs(reinterpret_cast<const float4 *>(row + cgl * 4))
                                       : make_float4(0.f, 0.f, 0.f, 0.f);
       }
@@ -160,7 +161,7 @@ logreg_fused_kernel(const LogregArgs p) {
     __syncthreads();
     Dots tot = red[buf][0];
 #pragma unroll
-    for (int w = 1; w < kLrWarps; ++w) dots_add(tot, red[buf][w]);
+    for (int w = 1; w < kWarps; ++w) dots_add(tot, red[buf][w]);
     if (CLUSTER) {
       // tot is this CTA's share (its column chunk).  Thread t hands it to the CTA of rank t;
       // after the barrier every CTA adds the shares in rank order.  Two buffers: a CTA can only
@@ -192,7 +193,7 @@ logreg_fused_kernel(const LogregArgs p) {
   float *out = p.partial + ((int64_t)i * p.P + blk) * p.d + cg0 * 4;
 #pragma unroll
   for (int j = 0; j < VPT; ++j) {
-    const int64_t cgl = threadIdx.x + (int64_t)j * kLrThreads;
+    const int64_t cgl = threadIdx.x + (int64_t)j * T;
     if (valid[j]) *reinterpret_cast<float4 *>(out + cgl * 4) = acc[j];
   }
 }
@@ -278,27 +279,30 @@ static ceca_status_t enqueue_grad(const float *A, const float *targets, const fl
     a.inv_m = inv_m;
     a.chunks = chunks;
     a.chunk4 = (d / 4 + chunks - 1) / chunks;
-    const int64_t groups = (a.chunk4 + kLrThreads - 1) / kLrThreads;   // float4 per thread and row
+    const int threads = a.chunk4 > (int64_t)kLrThreads * kLrMaxVpt ? 2 * kLrThreads : kLrThreads;
+    const int64_t groups = (a.chunk4 + threads - 1) / threads;   // float4 per thread and row
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)P * chunks, (unsigned)n);
-    cfg.blockDim = dim3(kLrThreads);
+    cfg.blockDim = dim3(threads);
     cfg.stream = stream;
     cudaLaunchAttribute attr;
     attr.id = cudaLaunchAttributeClusterDimension;
     attr.val.clusterDim.x = chunks; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
+    if (chunks > 1) { cfg.attrs = &attr; cfg.numAttrs = 1; }
     cudaError_t e;
-    if (chunks > 1) {
-      cfg.attrs = &attr; cfg.numAttrs = 1;
-      if (groups <= 1)      e = cudaLaunchKernelEx(&cfg, logreg_fused_kernel<1, LOSS, true>, a);
-      else if (groups <= 2) e = cudaLaunchKernelEx(&cfg, logreg_fused_kernel<2, LOSS, true>, a);
-      else if (groups <= 4) e = cudaLaunchKernelEx(&cfg, logreg_fused_kernel<4, LOSS, true>, a);
-      else                  e = cudaLaunchKernelEx(&cfg, logreg_fused_kernel<8, LOSS, true>, a);
+#define CECA_LR_LAUNCH(VPT_, CL_, T_) e = cudaLaunchKernelEx(&cfg, logreg_fused_kernel<VPT_, LOSS, CL_, T_>, a)
+    if (threads > kLrThreads) {
+      if (chunks > 1) CECA_LR_LAUNCH(4, true, 2 * kLrThreads); else CECA_LR_LAUNCH(4, false, 2 * kLrThreads);
+    } else if (chunks > 1) {
+      if (groups <= 1) CECA_LR_LAUNCH(1, true, kLrThreads);
+      else if (groups <= 2) CECA_LR_LAUNCH(2, true, kLrThreads);
+      else CECA_LR_LAUNCH(4, true, kLrThreads);
     } else {
-      if (groups <= 1)      e = cudaLaunchKernelEx(&cfg, logreg_fused_kernel<1, LOSS, false>, a);
-      else if (groups <= 2) e = cudaLaunchKernelEx(&cfg, logreg_fused_kernel<2, LOSS, false>, a);
-      else if (groups <= 4) e = cudaLaunchKernelEx(&cfg, logreg_fused_kernel<4, LOSS, false>, a);
-      else                  e = cudaLaunchKernelEx(&cfg, logreg_fused_kernel<8, LOSS, false>, a);
+      if (groups <= 1) CECA_LR_LAUNCH(1, false, kLrThreads);
+      else if (groups <= 2) CECA_LR_LAUNCH(2, false, kLrThreads);
+      else CECA_LR_LAUNCH(4, false, kLrThreads);
     }
+#undef CECA_LR_LAUNCH
     if (e != cudaSuccess) return CECA_ERR_CUDA;
     const int64_t work = (int64_t)n * (d / 4);
     logreg_reduce_kernel<<<(unsigned)((work + 255) / 256), 256, 0, stream>>>(partial, noise, G, n, P, d, ld);
