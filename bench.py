@@ -57,6 +57,9 @@ WORKLOADS = {
     "consensus_fused_smem": dict(kind="consensus", n=97, d=1 << 20, variant=2, fused=2),
     "consensus_fused_tmem": dict(kind="consensus", n=97, d=1 << 20, variant=2, fused=3),
     "consensus_rounds": dict(kind="consensus", n=97, d=1 << 20, variant=2, fused=0),
+    # the 1-port sequence (pairwise exchange, even n): fused and per round
+    "consensus_fused_1p": dict(kind="consensus", n=100, d=1 << 20, variant=1, fused=1),
+    "consensus_rounds_1p": dict(kind="consensus", n=100, d=1 << 20, variant=1, fused=0),
     # half the columns: the case the profiler captures are taken on (0.2 GB in, 0.4 GB out)
     "consensus_fused_small": dict(kind="consensus", n=97, d=1 << 19, variant=2, fused=1),
     # the paper's network sizes (Sec. 5): n = 130, n = 258 (32-column tiles) and n = 1026 (16-column tiles, eleven rounds)
@@ -88,12 +91,12 @@ FALLBACK_HBM_GBS = 6650.0
 NCU_TRAFFIC = {
     # 19.73 B per agent-parameter measured on step_small (2.5166 GB read + 1.6220 GB written for
     # 100 x 2,097,152 units); traffic is proportional to the units, scaled to n*d of resnet50_step
-    "step_small": (4.1386e9, "dram_traffic__step_consensus_gradient.md", "step.cu", "b16a43e291d9"),
-    "resnet50_step": (19.734 * 100 * 25_557_032, "dram_traffic__step_consensus_gradient.md", "step.cu", "b16a43e291d9"),
+    "step_small": (4.1386e9, "dram_traffic__step_consensus_gradient.md", "step.cu", "ceefd77ff7b3"),
+    "resnet50_step": (19.734 * 100 * 25_557_032, "dram_traffic__step_consensus_gradient.md", "step.cu", "ceefd77ff7b3"),
     # cycles of two rows (every CECA-1P round): 19.72 B per agent-parameter on step_small's round 6, scaled by units
-    "resnet18_step": (19.72 * 24 * 11_689_512, "dram_traffic__step_consensus_gradient.md", "step.cu", "b16a43e291d9"),
+    "resnet18_step": (19.72 * 24 * 11_689_512, "dram_traffic__step_consensus_gradient.md", "step.cu", "ceefd77ff7b3"),
     # seven launches of a cycle: round 0 moves 1.168 GB, the six others 1.565 GB each
-    "consensus_rounds": (10.558e9, "dram_traffic__step_consensus_gradient.md", "step.cu", "b16a43e291d9"),
+    "consensus_rounds": (10.558e9, "dram_traffic__step_consensus_gradient.md", "step.cu", "ceefd77ff7b3"),
     # fused kernel 2.0735 GB + fixed-order reduce 0.0299 GB
     "logreg_grad": (2.1034e9, "dram_traffic__step_consensus_gradient.md", "logreg.cu", "1bf7d97691f2"),
     "logreg_grad_d32768": (2.1357e9, "dram_traffic__step_consensus_gradient.md", "logreg.cu", "1bf7d97691f2"),
