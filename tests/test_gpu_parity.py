@@ -974,4 +974,29 @@ def test_heterogeneous_logreg_full_size_first_iterations(n, variant):
         ceca.ceca_gossip_sgd_step(X, Y, G, gamma, variant, k)
         want_x, want_y = oracle.step(bx, by, bg, np.float32(gamma), variant, k)
         tol = STEP_TOL * max(np.abs(bx).max(), np.abs(by).max(), gamma * np.abs(bg).max())
-        assert np.abs(_np(X) - want_x).max() <= tol and np.abs(_np(Y) - want_y).max() <= tol
+        assert np.abs(_np(X) - want_x).max() <= tol and np.abs(_np(Y) - want_y).max() <= tol@pytest.mark.gpu
+def test_register_block_consensus_over_the_whole_range_of_agent_counts():
+    """The register-block kernel picks its tile width, block size and launch shape from n: every n up to its
+    limit, with an odd width that ends in a lone column or a width of several tiles with a ragged last one, a
+    start at the beginning of a cycle (Y ignored) and one in the middle of it (Y read)."""
+    rng = np.random.default_rng(7)
+    for n in range(2, BLOCK_MAX_N + 1):
+        d = 37 if n % 2 else 130
+        x = synth.consensus_inputs(n, d, seed=n, offset_rows=False)
+        y = synth.consensus_inputs(n, d, seed=n + 1, offset_rows=False)
+        tau = _tau(n)
+        for k0, rounds in ((0, tau), (int(rng.integers(1, 3 * tau + 1)), int(rng.integers(1, tau + 3)))):
+            ws = _fused_ws()
+            ld = (d + 3) // 4 * 4 + 4     # padded rows, 16-byte aligned
+            Xo, Yo = torch.full((n, ld), float("nan"), device=DEV)[:, :d], torch.full((n, ld), float("nan"), device=DEV)[:, :d]
+            X = torch.empty((n, ld), device=DEV)[:, :d]; X.copy_(x)
+            Y = torch.empty((n, ld), device=DEV)[:, :d]; Y.copy_(y)
+            ceca.ceca_consensus_rounds(X, Y, ceca.CECA_2P, k0, rounds, ceca.FUSED_BLOCK, X_out=Xo, Y_out=Yo, workspace=ws)
+            assert ceca.ceca_read_status(ws) == 0
+            want_x, want_y = oracle.consensus(_np(x), _np(y), ceca.CECA_2P, k0, rounds)
+            tol = STEP_TOL * rounds * _scale(0, (x, 1), (y, 1))
+            assert np.abs(_np(Xo) - want_x).max() <= tol, (n, k0, rounds)
+            assert np.abs(_np(Yo) - want_y).max() <= tol, (n, k0, rounds)
+
+
+
