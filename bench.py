@@ -52,7 +52,7 @@ WORKLOADS = {
     "step_odd_ld": dict(kind="step", n=100, d=4_194_303, variant=2, gamma=0.1, ld=4_194_303),
     # n a power of two: the X-only update (12 B per agent-parameter; CECA-2P = one-peer exponential graph)
     "pow2_xonly_step": dict(kind="step", n=128, d=8_388_608, variant=2, gamma=0.1, x_only=True),
-    # fused = 1 picks the kernel by n and variant (register blocks for CECA-2P up to n = 1152, shared-memory exchange otherwise)
+    # fused = 1 picks the kernel by n and variant (register blocks for CECA-2P up to n = 1152 and CECA-1P up to n = 208)
     "consensus_fused": dict(kind="consensus", n=97, d=1 << 20, variant=2, fused=1),
     "consensus_fused_smem": dict(kind="consensus", n=97, d=1 << 20, variant=2, fused=2),
     "consensus_fused_tmem": dict(kind="consensus", n=97, d=1 << 20, variant=2, fused=3),
@@ -101,10 +101,10 @@ NCU_TRAFFIC = {
     "logreg_grad": (2.1034e9, "dram_traffic__step_consensus_gradient.md", "logreg.cu", "1bf7d97691f2"),
     "logreg_grad_d32768": (2.1357e9, "dram_traffic__step_consensus_gradient.md", "logreg.cu", "1bf7d97691f2"),
     # register-block kernel: captured at d = 2^19 (0.5522 GB per launch) and doubled for d = 2^20 (traffic is per tile)
-    "consensus_fused_small": (0.5522e9, "consensus_block_kernel__n97_n258_n1026__ncu_full.md", "consensus_block.cu", "45b50a63710f"),
-    "consensus_fused": (1.1044e9, "consensus_block_kernel__n97_n258_n1026__ncu_full.md", "consensus_block.cu", "45b50a63710f"),
-    "consensus_fused_258": (1.5641e9, "consensus_block_kernel__n97_n258_n1026__ncu_full.md", "consensus_block.cu", "45b50a63710f"),
-    "consensus_fused_1026": (3.1769e9, "consensus_block_kernel__n97_n258_n1026__ncu_full.md", "consensus_block.cu", "45b50a63710f"),
+    "consensus_fused_small": (0.5522e9, "consensus_block_kernel__n97_n258_n1026__ncu_full.md", "consensus_block.cu", "8a0c68ff353e"),
+    "consensus_fused": (1.1044e9, "consensus_block_kernel__n97_n258_n1026__ncu_full.md", "consensus_block.cu", "8a0c68ff353e"),
+    "consensus_fused_258": (1.5641e9, "consensus_block_kernel__n97_n258_n1026__ncu_full.md", "consensus_block.cu", "8a0c68ff353e"),
+    "consensus_fused_1026": (3.1769e9, "consensus_block_kernel__n97_n258_n1026__ncu_full.md", "consensus_block.cu", "8a0c68ff353e"),
 }
 
 
@@ -440,7 +440,7 @@ def bench_consensus(args, wl, device, dist):
         kernel = "step_walk_kernel<float4, no gradient> x tau"
     elif fused == 3:
         kernel = "consensus_tmem_kernel (tensor-memory exchange)"
-    elif fused == 2 or n > 1152 or variant != 2:
+    elif fused == 2 or n > (1152 if variant == 2 else 208):
         kernel = "consensus_fused_kernel (shared-memory exchange of every row)"
     else:
         kernel = "consensus_block_kernel (register blocks, boundary rows through shared memory)"

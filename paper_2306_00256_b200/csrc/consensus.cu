@@ -33,8 +33,8 @@ cudaError_t enqueue_step(const Plan &plan, const float *X, const float *Y, const
 ceca_status_t check_matrix_args(const void *X, const void *X_out, int32_t n, int64_t d, int64_t ld);
 bool consensus_block_supports(int32_t n, ceca_variant_t variant, int32_t rounds, bool y_in);
 ceca_status_t consensus_block(const float *X, const float *Y, float *Xo, float *Yo, int32_t n, int64_t d,
-                              int64_t ld, int64_t k0, int32_t rounds, int32_t *status, int32_t wait_polls,
-                              uint32_t tx_extra, int warps_override, cudaStream_t stream);
+                              int64_t ld, ceca_variant_t variant, int64_t k0, int32_t rounds, int32_t *status,
+                              int32_t wait_polls, uint32_t tx_extra, int warps_override, cudaStream_t stream);
 bool consensus_tmem_supports(int32_t n, int32_t rounds);
 ceca_status_t consensus_tmem(const float *X, const float *Y, float *Xo, float *Yo, int32_t n, int64_t d,
                              int64_t ld, ceca_variant_t variant, int64_t k0, int32_t rounds, int32_t *status,
@@ -272,7 +272,7 @@ static ceca_status_t consensus_fused(const float *X, const float *Y, float *Xo, 
   const bool block_ok = consensus_block_supports(n, variant, rounds, args.has_y_in != 0);
   if (kind == CECA_FUSED_BLOCK && !block_ok) return CECA_ERR_UNSUPPORTED;
   if (kind == CECA_FUSED_BLOCK || (kind == CECA_FUSED_AUTO && block_ok))
-    return consensus_block(X, args.has_y_in ? Y : nullptr, Xo, Yo, n, d, ld, k0, rounds, args.status, wait_polls,
+    return consensus_block(X, args.has_y_in ? Y : nullptr, Xo, Yo, n, d, ld, variant, k0, rounds, args.status, wait_polls,
                            tx_extra, 0, stream);
   if (kind == CECA_FUSED_TMEM)
     return consensus_tmem(X, args.has_y_in ? Y : nullptr, Xo, Yo, n, d, ld, variant, k0, rounds, args.status,

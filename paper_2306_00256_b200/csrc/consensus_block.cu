@@ -1,5 +1,5 @@
-// Fused CECA-2P consensus rounds (Sec. 3.1 "Main recursions", Algorithm 2) with register-resident
-// blocks of agents: most of every round's exchange never leaves the register file, and what the
+// Fused CECA consensus rounds (Sec. 3.1 "Main recursions", Algorithm 2; the 1-port pairing of Sec. 3.2
+// further down) with register-resident blocks of agents: most of every round's exchange never leaves the register file, and what the
 // kernel executes per value and round is close to the one fused multiply-add it has to do.
 //
 // Layout.  A CTA owns one column tile of all n rows (TMA tensor loads into shared memory).  A thread
@@ -143,6 +143,7 @@ __device__ __forceinline__ void sts64(uint32_t addr, pk2 v) {
 struct BlockPos {
   uint32_t own;    // row i0 of the exchange tile
   uint32_t prev;   // in-register rounds: the row just after the S source rows (row i0; row n for block 0)
+  uint32_t next;   // 1-port rounds: the first row after the block (row 0 for the last block)
   uint32_t col;    // row 0
   int i0, cnt;     // cnt = real rows of the block (CB, fewer in the last block)
   bool full, publish;
@@ -251,10 +252,125 @@ __device__ __forceinline__ void dispatch_round(int sel, int s, int n, pk2 (&Ih)[
 #undef CECA_BK_CASE
 }
 
+// ---- CECA-1P (Sec. 3.2): pairwise exchange -------------------------------------------------------
+// Round r pairs even row i with row i + o, o = 2 n_r + 1 (odd, modulo the even n): even rows receive
+// from o rows further on, odd rows from o rows back, and the two rows of a pair swap their payloads.
+// Blocks hold an even number of agents and start at even rows (sizes CB and CB - 2), so parity is a
+// property of the register position: position 2p is an even row ("E_p"), 2p + 1 an odd one ("O_p").
+// With h = n_r the pairing reads E_p <-> O_{p+h}: while h is smaller than a block, the pairs whose two
+// rows lie in the same block swap in registers, the last h even rows of a block pair with the first h
+// odd rows of the next one, and only those 2 h rows per block go through shared memory.
+
+// One 1-port round with compile-time h = H smaller than every block (in pairs).
+template <int CB, int RB, int CH, int H, bool PAYJ>
+__device__ __forceinline__ void round_partial_1p(pk2 (&Ih)[CB], pk2 (&Jh)[CB], pk2 cI, pk2 cJ, const BlockPos &q) {
+  constexpr int C = CB / 2;   // pairs of positions in a full block; a short block has C - 1
+  pk2(&Z)[CB] = PAYJ ? Jh : Ih;
+  if constexpr (H > 0) {
+    if (q.publish) {
+      // the odd rows of the first H pairs (wanted by the block before) and the even rows of the last H pairs
+      static_for<H>([&](auto T) { sts64<(2 * CECA_IDX(T) + 1) * RB>(q.own, Z[2 * CECA_IDX(T) + 1]); });
+      if (q.full) {
+        static_for<H>([&](auto T) { sts64<2 * (C - H + CECA_IDX(T)) * RB>(q.own, Z[2 * (C - H + CECA_IDX(T))]); });
+      } else if constexpr (C - 1 - H >= 0) {
+        static_for<H>([&](auto T) { sts64<2 * (C - 1 - H + CECA_IDX(T)) * RB>(q.own, Z[2 * (C - 1 - H + CECA_IDX(T))]); });
+      }
+      __syncthreads();
+    }
+  }
+  // pairs inside the block: both rows read the other's value from before the round
+  static_for<C - H>([&](auto P) {
+    constexpr int e = 2 * CECA_IDX(P), o = 2 * (CECA_IDX(P) + H) + 1;
+    if (q.full || CECA_IDX(P) < C - 1 - H) {   // in a short block the last pair of positions is not there
+      const pk2 ze = Z[e], zo = Z[o];
+      Ih[e] = axpy2(cI, zo, Ih[e]); Jh[e] = axpy2(cJ, zo, Jh[e]);
+      Ih[o] = axpy2(cI, ze, Ih[o]); Jh[o] = axpy2(cJ, ze, Jh[o]);
+    }
+  });
+  if constexpr (H > 0) {
+    // the first H odd rows receive from the even rows 2 H - 1, 2 H - 3, ... rows before them (previous block)
+    static_for<H>([&](auto T) {
+      constexpr int o = 2 * CECA_IDX(T) + 1;
+      const pk2 r = lds64<2 * (CECA_IDX(T) - H) * RB>(q.prev);
+      Ih[o] = axpy2(cI, r, Ih[o]); Jh[o] = axpy2(cJ, r, Jh[o]);
+    });
+    // the last H even rows receive from the first H odd rows of the next block
+    if (q.full) {
+      static_for<H>([&](auto T) {
+        constexpr int e = 2 * (C - H + CECA_IDX(T));
+        const pk2 r = lds64<(2 * CECA_IDX(T) + 1) * RB>(q.next);
+        Ih[e] = axpy2(cI, r, Ih[e]); Jh[e] = axpy2(cJ, r, Jh[e]);
+      });
+    } else if constexpr (C - 1 - H >= 0) {
+      static_for<H>([&](auto T) {
+        constexpr int e = 2 * (C - 1 - H + CECA_IDX(T));
+        const pk2 r = lds64<(2 * CECA_IDX(T) + 1) * RB>(q.next);
+        Ih[e] = axpy2(cI, r, Ih[e]); Jh[e] = axpy2(cJ, r, Jh[e]);
+      });
+    }
+  }
+}
+
+// One 1-port round in which every row receives through shared memory (h at least as large as a block).
+template <int CB, int RB, bool PAYJ>
+__device__ __forceinline__ void round_full_1p(pk2 (&Ih)[CB], pk2 (&Jh)[CB], pk2 cI, pk2 cJ, const BlockPos &q, int o, int n) {
+  pk2(&Z)[CB] = PAYJ ? Jh : Ih;
+  if (q.publish) {
+    static_for<CB - 2>([&](auto J) { sts64<CECA_IDX(J) * RB>(q.own, Z[CECA_IDX(J)]); });
+    if (q.full) { sts64<(CB - 2) * RB>(q.own, Z[CB - 2]); sts64<(CB - 1) * RB>(q.own, Z[CB - 1]); }
+    __syncthreads();
+  }
+  // even rows read o rows further on, odd rows o rows back; each of the two streams is contiguous
+  // unless the wrap-around at n falls inside it
+  int fe = q.i0 + o, fo = q.i0 - o;
+  const bool e_plain = fe + q.cnt <= n || fe >= n, o_plain = fo >= 0 || fo + q.cnt <= 0;
+  if (fe >= n) fe -= n;
+  if (fo + q.cnt <= 0) fo += n;
+  if (e_plain && o_plain) {
+    const uint32_t se = q.col + (uint32_t)(fe * RB), so = q.col + (uint32_t)(fo * RB);
+    static_for<CB>([&](auto J) {
+      constexpr int j = CECA_IDX(J);
+      const pk2 r = (j < CB - 2 || q.full) ? lds64<j * RB>((j & 1) ? so : se) : 0ull;
+      Ih[j] = axpy2(cI, r, Ih[j]); Jh[j] = axpy2(cJ, r, Jh[j]);
+    });
+  } else {
+#pragma unroll
+    for (int j = 0; j < CB; ++j) {
+      int row = (j & 1) ? q.i0 + j - o : q.i0 + j + o;
+      if (row < 0) row += n;
+      if (row >= n) row -= n;
+      const pk2 r = (j < q.cnt) ? lds64<0>(q.col + (uint32_t)(row * RB)) : 0ull;
+      Ih[j] = axpy2(cI, r, Ih[j]); Jh[j] = axpy2(cJ, r, Jh[j]);
+    }
+  }
+}
+
+// `sel`: 0 / 1 = every row through shared memory, payload I / J; 2 (H + 1) + (0 / 1) = the in-register form.
+template <int CB, int RB, int CH>
+__device__ __forceinline__ void dispatch_round_1p(int sel, int o, int n, pk2 (&Ih)[CB], pk2 (&Jh)[CB], pk2 cI, pk2 cJ,
+                                                  const BlockPos &q) {
+#define CECA_BK_CASE(H)                                                                   \
+  case 2 * (H + 1):                                                                       \
+    if constexpr (H < CB / 2) round_partial_1p<CB, RB, CH, H, false>(Ih, Jh, cI, cJ, q);  \
+    break;                                                                                \
+  case 2 * (H + 1) + 1:                                                                   \
+    if constexpr (H < CB / 2) round_partial_1p<CB, RB, CH, H, true>(Ih, Jh, cI, cJ, q);   \
+    break;
+  switch (sel) {
+    case 0: round_full_1p<CB, RB, false>(Ih, Jh, cI, cJ, q, o, n); break;
+    case 1: round_full_1p<CB, RB, true>(Ih, Jh, cI, cJ, q, o, n); break;
+    CECA_BK_CASE(0) CECA_BK_CASE(1) CECA_BK_CASE(2) CECA_BK_CASE(3) CECA_BK_CASE(4) CECA_BK_CASE(5) CECA_BK_CASE(6)
+    CECA_BK_CASE(7) CECA_BK_CASE(8) CECA_BK_CASE(9) CECA_BK_CASE(10) CECA_BK_CASE(11) CECA_BK_CASE(12)
+    default: break;
+  }
+#undef CECA_BK_CASE
+}
+
 // CB agents per block, LPB threads (column pairs) per block.  The number of threads per CTA is a
 // launch parameter; MAXT only bounds it and thereby sets the register budget (65536 / MAXT registers
 // per thread).
-template <int CB, int LPB, int MAXT>
+// ONEP: the CECA-1P form (blocks of CB or CB - 2 agents, CB even; 64-column tiles only).
+template <int CB, int LPB, int MAXT, bool ONEP>
 __global__ void __launch_bounds__(MAXT, 1)
 consensus_block_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_y,
                        const __grid_constant__ BlockArgs p) {
@@ -275,7 +391,11 @@ consensus_block_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
   const uint32_t y_tile = p.single_xch ? 2u : 3u;
 
   BlockPos q;
-  if (kBalanced) {
+  if (ONEP) {   // pairs of rows: the first p.nfull blocks hold CB / 2 of them, the others one less
+    q.full = part < p.nfull;
+    q.cnt = q.full ? CB : CB - 2;
+    q.i0 = q.full ? part * CB : p.nfull * CB + (part - p.nfull) * (CB - 2);
+  } else if (kBalanced) {
     q.full = part < p.nfull;
     q.cnt = q.full ? CB : CB - 1;
     q.i0 = q.full ? part * CB : p.nfull * CB + (part - p.nfull) * (CB - 1);
@@ -287,6 +407,8 @@ consensus_block_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
   const uint32_t col_off = 2u * lane * (uint32_t)sizeof(float);
   const uint32_t own_off = (uint32_t)q.i0 * RB + col_off;
   const uint32_t prev_off = (uint32_t)(part == 0 ? n : q.i0) * RB + col_off;
+  // 1-port: the row after the block's last one (the last block is followed by row 0)
+  const uint32_t next_off = (ONEP && part < p.blocks - 1) ? own_off + (uint32_t)q.cnt * RB : col_off;
 
   if (threadIdx.x == 0) {
     mbar_init(&bar, 1);
@@ -329,7 +451,7 @@ consensus_block_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
       } else {
         static_for<CB>([&](auto J) {
           constexpr int j = CECA_IDX(J);
-          if constexpr (kBalanced && j < CB - 1) Ih[j] = lds64<j * RB>(own);
+          if constexpr (kBalanced && j < CB - (ONEP ? 2 : 1)) Ih[j] = lds64<j * RB>(own);
           else Ih[j] = (q.full || j < q.cnt) ? lds64<j * RB>(own) : 0ull;
         });
       }
@@ -341,7 +463,7 @@ consensus_block_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
       } else {
         static_for<CB>([&](auto J) {
           constexpr int j = CECA_IDX(J);
-          if constexpr (kBalanced && j < CB - 1) Jh[j] = lds64<j * RB>(owny);
+          if constexpr (kBalanced && j < CB - (ONEP ? 2 : 1)) Jh[j] = lds64<j * RB>(owny);
           else Jh[j] = (q.full || j < q.cnt) ? lds64<j * RB>(owny) : 0ull;
         });
       }
@@ -374,7 +496,12 @@ consensus_block_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
       q.own = buf + own_off;
       q.prev = buf + prev_off;
       q.col = buf + col_off;
-      dispatch_round<CB, RB, kBalanced, kInFlight>(rd.sel, rd.hop, p.n, Ih, Jh, pk_make(rd.cI, rd.cI), pk_make(rd.cJ, rd.cJ), q);
+      if constexpr (ONEP) {
+        q.next = buf + next_off;
+        dispatch_round_1p<CB, RB, kInFlight>(rd.sel, rd.hop, p.n, Ih, Jh, pk_make(rd.cI, rd.cI), pk_make(rd.cJ, rd.cJ), q);
+      } else {
+        dispatch_round<CB, RB, kBalanced, kInFlight>(rd.sel, rd.hop, p.n, Ih, Jh, pk_make(rd.cI, rd.cI), pk_make(rd.cJ, rd.cJ), q);
+      }
       // with a single exchange tile the next round's publish must wait for this round's reads
       if (p.single_xch && rnd >= 1 && rnd + 1 < p.rounds) __syncthreads();
     }
@@ -396,12 +523,12 @@ consensus_block_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
       } else {
         static_for<CB>([&](auto J) {
           constexpr int j = CECA_IDX(J);
-          if ((kBalanced && j < CB - 1) || q.full || j < q.cnt) __stcs(reinterpret_cast<pk2 *>(dst + j * p.ld), mul2(oI, Ih[j]));
+          if ((kBalanced && j < CB - (ONEP ? 2 : 1)) || q.full || j < q.cnt) __stcs(reinterpret_cast<pk2 *>(dst + j * p.ld), mul2(oI, Ih[j]));
         });
         if (p.has_y_out) {
           static_for<CB>([&](auto J) {
             constexpr int j = CECA_IDX(J);
-            if ((kBalanced && j < CB - 1) || q.full || j < q.cnt) __stcs(reinterpret_cast<pk2 *>(dsty + j * p.ld), mul2(oJ, Jh[j]));
+            if ((kBalanced && j < CB - (ONEP ? 2 : 1)) || q.full || j < q.cnt) __stcs(reinterpret_cast<pk2 *>(dsty + j * p.ld), mul2(oJ, Jh[j]));
           });
         }
       }
@@ -449,6 +576,19 @@ struct BlockGeom {
 };
 constexpr int kBkMaxRows = 1152;
 constexpr int kBkPlain = 0, kBkCompact = 1;
+constexpr int kBkMaxRows1p = 208;   // CECA-1P: eight warps of 26 agents
+// CECA-1P: n / 2 pairs of rows in 1, 2, 4 or 8 blocks (warps) of C or C - 1 pairs; cb = 2 C, cmin in pairs.
+static bool block_geometry_1p(int n, BlockGeom *g) {
+  if (n < 2 || (n & 1) || n > kBkMaxRows1p) return false;
+  const int pairs = n / 2;
+  int blocks = n <= 26 ? 1 : n <= 52 ? 2 : n <= 104 ? 4 : 8;
+  if (blocks > pairs) blocks = pairs;
+  const int c = (pairs + blocks - 1) / blocks;
+  g->lpb = 32; g->blocks = blocks; g->cb = 2 * c; g->threads = 32 * blocks;
+  g->nfull = pairs - blocks * (c - 1);
+  g->cmin = g->nfull == blocks ? c : c - 1;
+  return g->cb <= 26;
+}
 static bool block_geometry(int n, int warps_override, int kind, BlockGeom *g) {
   if (n < 2 || n > kBkMaxRows) return false;
   if (n <= 400) {
@@ -508,7 +648,12 @@ static BlockTile block_tile(int n, const BlockGeom &g) {
 
 // y_in: the first round reads Y, which takes one more shared-memory tile (at least two are needed without it).
 bool consensus_block_supports(int32_t n, ceca_variant_t variant, int32_t rounds, bool y_in) {
-  if (variant != CECA_2P || rounds < 1 || rounds > kBkMaxRounds) return false;
+  if (rounds < 1 || rounds > kBkMaxRounds) return false;
+  if (variant == CECA_1P) {
+    BlockGeom g;
+    return block_geometry_1p(n, &g) && (size_t)(y_in ? 3 : 2) * block_tile(n, g).tile_bytes <= kBkSmemLimit;
+  }
+  if (variant != CECA_2P) return false;
   for (int kind = 0; kind < 2; ++kind) {
     BlockGeom g;
     if (block_geometry(n, 0, kind, &g) && (size_t)(y_in ? 3 : 2) * block_tile(n, g).tile_bytes <= kBkSmemLimit) return true;
@@ -520,18 +665,18 @@ bool consensus_block_supports(int32_t n, ceca_variant_t variant, int32_t rounds,
 // still compiles without spilling to speak of.  65536 / kMaxThreads registers per thread.
 template <int CB> struct BlockRegs {
   static constexpr int kRoomy = CB >= 15 ? 384 : CB >= 11 ? 640 : CB >= 7 ? 768 : 1024;
-  static constexpr int kLean = CB >= 15 ? 512 : CB >= 11 ? 768 : 1024;
+  static constexpr int kLean = CB >= 26 ? 384 : CB >= 15 ? 512 : CB >= 11 ? 768 : 1024;
 };
 
-template <int CB, int LPB, int MAXT>
+template <int CB, int LPB, int MAXT, bool ONEP>
 static cudaError_t launch_block_regs(const CUtensorMap *maps, const BlockArgs &a, int threads,
                                      size_t smem, int *per_sm_out, bool launch, cudaStream_t stream) {
   static std::atomic<uint64_t> attr_done{0};
-  cudaError_t e = set_max_shared_once(reinterpret_cast<const void *>(consensus_block_kernel<CB, LPB, MAXT>),
+  cudaError_t e = set_max_shared_once(reinterpret_cast<const void *>(consensus_block_kernel<CB, LPB, MAXT, ONEP>),
                                       kBkSmemLimit, &attr_done);
   if (e != cudaSuccess) return e;
   int per_sm = 0;
-  e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, consensus_block_kernel<CB, LPB, MAXT>, threads, smem);
+  e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, consensus_block_kernel<CB, LPB, MAXT, ONEP>, threads, smem);
   if (e != cudaSuccess) return e;
   *per_sm_out = per_sm;
   if (!launch) return cudaSuccess;
@@ -541,18 +686,23 @@ static cudaError_t launch_block_regs(const CUtensorMap *maps, const BlockArgs &a
   // persistent CTAs: as many as fit on the device at once, not more than there are tiles
   const int64_t resident = (int64_t)sms * per_sm;
   const int grid = (int)(a.tiles < resident ? a.tiles : resident);
-  consensus_block_kernel<CB, LPB, MAXT><<<grid, threads, smem, stream>>>(maps[0], maps[1], a);
+  consensus_block_kernel<CB, LPB, MAXT, ONEP><<<grid, threads, smem, stream>>>(maps[0], maps[1], a);
   return cudaGetLastError();
 }
 
 // launch == false: only reports in *ctas_per_sm how many CTAs of the best launch shape share an SM.
-template <int CB, int LPB>
+template <int CB, int LPB, bool ONEP>
 static cudaError_t launch_block(const CUtensorMap *maps, BlockArgs &a, int threads, int cmin, bool launch,
                                 int *ctas_per_sm, cudaStream_t stream) {
   for (int t = 0; t < a.rounds; ++t) {
     BlockRound &r = a.rd[t];
     const int pay = (r.mode & kBkPayloadJ) ? 1 : 0;
-    r.sel = r.hop < cmin ? 2 * r.hop + pay : pay;   // in-register form while the shift is smaller than every block
+    if (ONEP) {   // hop = 2 h + 1; cmin counts pairs of rows
+      const int h = (r.hop - 1) / 2;
+      r.sel = h < cmin ? 2 * (h + 1) + pay : pay;
+    } else {
+      r.sel = r.hop < cmin ? 2 * r.hop + pay : pay;   // in-register form while the shift is smaller than every block
+    }
   }
   const size_t tile_bytes = a.tile_bytes;
   // Four candidates: two or one exchange tile, roomy or lean register budget.  The default is two tiles
@@ -564,11 +714,11 @@ static cudaError_t launch_block(const CUtensorMap *maps, BlockArgs &a, int threa
     if (smem > kBkSmemLimit) continue;
     int roomy = 0, lean = 0;
     if (threads <= kRoomy) {
-      cudaError_t e = launch_block_regs<CB, LPB, kRoomy>(maps, a, threads, smem, &roomy, false, stream);
+      cudaError_t e = launch_block_regs<CB, LPB, kRoomy, ONEP>(maps, a, threads, smem, &roomy, false, stream);
       if (e != cudaSuccess) return e;
     }
     if (kLean != kRoomy && threads <= kLean) {
-      cudaError_t e = launch_block_regs<CB, LPB, kLean>(maps, a, threads, smem, &lean, false, stream);
+      cudaError_t e = launch_block_regs<CB, LPB, kLean, ONEP>(maps, a, threads, smem, &lean, false, stream);
       if (e != cudaSuccess) return e;
     }
     if (roomy > best) { best = roomy; best_single = single; best_lean = 0; }
@@ -580,17 +730,18 @@ static cudaError_t launch_block(const CUtensorMap *maps, BlockArgs &a, int threa
   a.single_xch = best_single;
   const size_t smem = ((a.has_y_in ? 2 : 1) + (best_single ? 1 : 2)) * tile_bytes;
   int per_sm = 0;
-  if (best_lean) return launch_block_regs<CB, LPB, kLean>(maps, a, threads, smem, &per_sm, true, stream);
-  return launch_block_regs<CB, LPB, kRoomy>(maps, a, threads, smem, &per_sm, true, stream);
+  if (best_lean) return launch_block_regs<CB, LPB, kLean, ONEP>(maps, a, threads, smem, &per_sm, true, stream);
+  return launch_block_regs<CB, LPB, kRoomy, ONEP>(maps, a, threads, smem, &per_sm, true, stream);
 }
 
 // Fills the geometry-dependent launch arguments for candidate `kind` and either launches it or only
 // reports its CTAs per SM.  CECA_ERR_UNSUPPORTED: this candidate does not exist for n or does not fit.
 static ceca_status_t block_dispatch(const float *X, const float *Y, float *Xo, float *Yo, int32_t n, int64_t d, int64_t ld,
-                                    BlockArgs &a, int kind, int warps_override, uint32_t tx_extra, bool launch,
-                                    int *ctas_per_sm, cudaStream_t stream) {
+                                    BlockArgs &a, bool one_port, int kind, int warps_override, uint32_t tx_extra,
+                                    bool launch, int *ctas_per_sm, cudaStream_t stream) {
   BlockGeom g;
-  if (!block_geometry(n, warps_override, kind, &g)) return CECA_ERR_UNSUPPORTED;
+  if (one_port ? (kind != kBkPlain || !block_geometry_1p(n, &g)) : !block_geometry(n, warps_override, kind, &g))
+    return CECA_ERR_UNSUPPORTED;
   const BlockTile t = block_tile(n, g);
   if ((size_t)(a.has_y_in ? 3 : 2) * t.tile_bytes > kBkSmemLimit) return CECA_ERR_UNSUPPORTED;
   const int tile_cols = 2 * g.lpb;
@@ -606,7 +757,19 @@ static ceca_status_t block_dispatch(const float *X, const float *Y, float *Xo, f
   }
 
   cudaError_t e = cudaErrorInvalidConfiguration;
-#define CECA_BK_LAUNCH(CB) case CB: e = launch_block<CB, kLpb>(maps, a, g.threads, g.cmin, launch, ctas_per_sm, stream); break;
+  if (one_port) {
+#define CECA_BK_LAUNCH(CB) case CB: e = launch_block<CB, 32, true>(maps, a, g.threads, g.cmin, launch, ctas_per_sm, stream); break;
+    switch (g.cb) {
+      CECA_BK_LAUNCH(2) CECA_BK_LAUNCH(4) CECA_BK_LAUNCH(6) CECA_BK_LAUNCH(8) CECA_BK_LAUNCH(10) CECA_BK_LAUNCH(12)
+      CECA_BK_LAUNCH(14) CECA_BK_LAUNCH(16) CECA_BK_LAUNCH(18) CECA_BK_LAUNCH(20) CECA_BK_LAUNCH(22) CECA_BK_LAUNCH(24)
+      CECA_BK_LAUNCH(26)
+      default: break;
+    }
+#undef CECA_BK_LAUNCH
+    if (e == cudaErrorInvalidConfiguration) return CECA_ERR_UNSUPPORTED;
+    return e == cudaSuccess ? CECA_OK : CECA_ERR_CUDA;
+  }
+#define CECA_BK_LAUNCH(CB) case CB: e = launch_block<CB, kLpb, false>(maps, a, g.threads, g.cmin, launch, ctas_per_sm, stream); break;
   if (g.lpb == 32) {
     constexpr int kLpb = 32;
     switch (g.cb) {
@@ -642,8 +805,9 @@ static ceca_status_t block_dispatch(const float *X, const float *Y, float *Xo, f
 // The caller has checked consensus_block_supports.  `warps_override` > 0 forces the number of
 // blocks for n <= 150 (used to measure the alternatives).
 ceca_status_t consensus_block(const float *X, const float *Y, float *Xo, float *Yo, int32_t n, int64_t d,
-                              int64_t ld, int64_t k0, int32_t rounds, int32_t *status, int32_t wait_polls,
-                              uint32_t tx_extra, int warps_override, cudaStream_t stream) {
+                              int64_t ld, ceca_variant_t variant, int64_t k0, int32_t rounds, int32_t *status,
+                              int32_t wait_polls, uint32_t tx_extra, int warps_override, cudaStream_t stream) {
+  const bool one_port = variant == CECA_1P;
   BlockArgs a;
   std::memset(&a, 0, sizeof(a));
   a.Xo = Xo; a.Yo = Yo; a.ld = ld; a.d = (int32_t)d; a.n = n; a.rounds = rounds;
@@ -655,7 +819,7 @@ ceca_status_t consensus_block(const float *X, const float *Y, float *Xo, float *
   bool first_needs_y = false;
   for (int32_t t = 0; t < rounds; ++t) {
     Plan plan;
-    ceca_status_t st = make_plan(n, CECA_2P, k0 + t, &plan);
+    ceca_status_t st = make_plan(n, variant, k0 + t, &plan);
     if (st != CECA_OK) return st;
     if (t == 0) first_needs_y = plan.reads_y;
     BlockRound &r = a.rd[t];
@@ -675,19 +839,19 @@ ceca_status_t consensus_block(const float *X, const float *Y, float *Xo, float *
   }
   a.outI = (float)alpha; a.outJ = (float)beta;
   a.has_y_in = (Y != nullptr && first_needs_y) ? 1 : 0;
-  if (!consensus_block_supports(n, CECA_2P, rounds, a.has_y_in != 0)) return CECA_ERR_UNSUPPORTED;
+  if (!consensus_block_supports(n, variant, rounds, a.has_y_in != 0)) return CECA_ERR_UNSUPPORTED;
 
   // The candidate geometries are asked how many CTAs they put on an SM; the first of the best is launched.
   int best_kind = -1, best_ctas = 0;
   for (int kind = 1; kind >= 0; --kind) {   // the compact candidate first: it wins ties
     int ctas = 0;
-    const ceca_status_t st = block_dispatch(X, Y, Xo, Yo, n, d, ld, a, kind, warps_override, tx_extra, false, &ctas, stream);
+    const ceca_status_t st = block_dispatch(X, Y, Xo, Yo, n, d, ld, a, one_port, kind, warps_override, tx_extra, false, &ctas, stream);
     if (st == CECA_OK && ctas > best_ctas) { best_ctas = ctas; best_kind = kind; }
     else if (st != CECA_OK && st != CECA_ERR_UNSUPPORTED) return st;
   }
   if (best_kind < 0) return CECA_ERR_UNSUPPORTED;
   int ctas = 0;
-  return block_dispatch(X, Y, Xo, Yo, n, d, ld, a, best_kind, warps_override, tx_extra, true, &ctas, stream);
+  return block_dispatch(X, Y, Xo, Yo, n, d, ld, a, one_port, best_kind, warps_override, tx_extra, true, &ctas, stream);
 }
 
 }  // namespace ceca

@@ -276,6 +276,7 @@ def test_mean_lemma_and_resume_on_gpu(n, variant):
 # --------------------------------------------------------------------------------------------
 
 BLOCK_MAX_N = 1152   # largest n the register-block kernel takes (16-column tiles of all rows on one SM)
+BLOCK_MAX_N_1P = 208  # ... with the 1-port pairing (eight warps of 26 agents)
 
 
 def _fused_ws():
@@ -284,11 +285,11 @@ def _fused_ws():
 
 def _fused_kernels(n, variant=ceca.CECA_2P):
     """The fused kernels that take n agents and this variant: shared-memory exchange (n <= 2048),
-    tensor-memory exchange (n <= 128), register blocks (CECA-2P, n <= 1152)."""
+    tensor-memory exchange (n <= 128), register blocks (CECA-2P: n <= 1152; CECA-1P: n <= 208)."""
     kernels = [ceca.FUSED_SMEM]
     if n <= 128:
         kernels.append(ceca.FUSED_TMEM)
-    if n <= BLOCK_MAX_N and variant == ceca.CECA_2P:
+    if n <= (BLOCK_MAX_N if variant == ceca.CECA_2P else BLOCK_MAX_N_1P):
         kernels.append(ceca.FUSED_BLOCK)
     return kernels
 
@@ -306,7 +307,7 @@ def test_consensus_matches_oracle_and_reaches_the_mean(fused, n, d):
     y0 = synth.consensus_inputs(n, d, seed=n + d + 1, offset_rows=False)
     tau = _tau(n)
     for variant in _variants(n):
-        if fused == ceca.FUSED_BLOCK and variant != ceca.CECA_2P:
+        if fused == ceca.FUSED_BLOCK and fused not in _fused_kernels(n, variant):
             continue
         for k0, rounds in [(0, tau), (0, tau + 1), (0, 1), (1 % tau, 2 * tau + 3), (5 * tau, tau)]:
             X, Y = x.to(DEV), y0.to(DEV)
@@ -440,7 +441,7 @@ def test_fused_consensus_many_rounds(fused):
     x = synth.consensus_inputs(n, d, seed=3)
     y = synth.consensus_inputs(n, d, seed=4, offset_rows=False)
     for variant in (ceca.CECA_2P, ceca.CECA_1P):
-        if fused == ceca.FUSED_BLOCK and variant != ceca.CECA_2P:
+        if fused == ceca.FUSED_BLOCK and fused not in _fused_kernels(n, variant):
             continue
         Xo, Yo = torch.empty(n, d, device=DEV), torch.empty(n, d, device=DEV)
         ws = _fused_ws()
@@ -460,7 +461,7 @@ def test_fused_consensus_padded_rows(fused):
     (X, xb), (Xo, xob), (Yo, yob) = _put(x.to(DEV), ld), _padded(n, d, ld), _padded(n, d, ld)
     ws = _fused_ws()
     for variant in (ceca.CECA_2P, ceca.CECA_1P):
-        if fused == ceca.FUSED_BLOCK and variant != ceca.CECA_2P:
+        if fused == ceca.FUSED_BLOCK and fused not in _fused_kernels(n, variant):
             continue
         ceca.ceca_consensus_rounds(X, None, variant, 0, 7, fused, X_out=Xo, Y_out=Yo, workspace=ws)
         want_x, want_y = oracle.consensus(_np(x), np.zeros((n, d)), variant, 0, 7)
@@ -825,7 +826,8 @@ def test_device_entry_points_reject_bad_arguments_and_launch_nothing():
     assert cons(x, None, xo, None, 6, 8, 8, 2, 0, 2, 0, None, 0, stream) == 5      # no Y_out, no workspace (n not 2^tau)
     assert cons(x, None, xo, None, 2050, 8, 8, 2, 0, 2, 1, ws, 256, stream) == 4   # n > 2048 fused
     assert cons(x, None, xo, None, 200, 8, 8, 2, 0, 2, 3, ws, 256, stream) == 4    # tensor-memory kernel: n <= 128
-    assert cons(x, None, xo, None, 6, 8, 8, 1, 0, 2, 4, ws, 256, stream) == 4      # register-block kernel: 2-port only
+    assert cons(x, None, xo, None, 210, 8, 8, 1, 0, 2, 4, ws, 256, stream) == 4    # register-block kernel: 1-port up to n = 208
+    assert cons(x, None, xo, None, 1154, 8, 8, 2, 0, 2, 4, ws, 256, stream) == 4   # ... 2-port up to n = 1152
     assert cons(x, None, xo, None, 4, 8, 8, 2, 0, 2, 7, ws, 256, stream) == 1      # no such kernel
     assert cons(x, None, xo_off, None, 4, 8, 8, 2, 0, 2, 1, ws, 256, stream) == 3  # misaligned
     assert cons(x, None, xo, None, 4, 8, 6, 2, 0, 2, 1, ws, 256, stream) == 1      # ld < d
@@ -974,29 +976,30 @@ def test_heterogeneous_logreg_full_size_first_iterations(n, variant):
         ceca.ceca_gossip_sgd_step(X, Y, G, gamma, variant, k)
         want_x, want_y = oracle.step(bx, by, bg, np.float32(gamma), variant, k)
         tol = STEP_TOL * max(np.abs(bx).max(), np.abs(by).max(), gamma * np.abs(bg).max())
-        assert np.abs(_np(X) - want_x).max() <= tol and np.abs(_np(Y) - want_y).max() <= tol@pytest.mark.gpu
+        assert np.abs(_np(X) - want_x).max() <= tol and np.abs(_np(Y) - want_y).max() <= tol
+
+
 def test_register_block_consensus_over_the_whole_range_of_agent_counts():
     """The register-block kernel picks its tile width, block size and launch shape from n: every n up to its
     limit, with an odd width that ends in a lone column or a width of several tiles with a ragged last one, a
     start at the beginning of a cycle (Y ignored) and one in the middle of it (Y read)."""
     rng = np.random.default_rng(7)
-    for n in range(2, BLOCK_MAX_N + 1):
-        d = 37 if n % 2 else 130
+    cases = [(n, ceca.CECA_2P) for n in range(2, BLOCK_MAX_N + 1)] + [(n, ceca.CECA_1P) for n in range(2, BLOCK_MAX_N_1P + 1, 2)]
+    for n, variant in cases:
+        d = 37 if (n // 2) % 2 else 130
         x = synth.consensus_inputs(n, d, seed=n, offset_rows=False)
         y = synth.consensus_inputs(n, d, seed=n + 1, offset_rows=False)
         tau = _tau(n)
-        for k0, rounds in ((0, tau), (int(rng.integers(1, 3 * tau + 1)), int(rng.integers(1, tau + 3)))):
+        for k0, rounds in ((0, tau), (int(rng.integers(1, 3 * tau + 1)), int(rng.integers(1, tau + 3))),
+                           (int(rng.integers(0, 3 * tau + 1)), 1)):
             ws = _fused_ws()
             ld = (d + 3) // 4 * 4 + 4     # padded rows, 16-byte aligned
             Xo, Yo = torch.full((n, ld), float("nan"), device=DEV)[:, :d], torch.full((n, ld), float("nan"), device=DEV)[:, :d]
             X = torch.empty((n, ld), device=DEV)[:, :d]; X.copy_(x)
             Y = torch.empty((n, ld), device=DEV)[:, :d]; Y.copy_(y)
-            ceca.ceca_consensus_rounds(X, Y, ceca.CECA_2P, k0, rounds, ceca.FUSED_BLOCK, X_out=Xo, Y_out=Yo, workspace=ws)
+            ceca.ceca_consensus_rounds(X, Y, variant, k0, rounds, ceca.FUSED_BLOCK, X_out=Xo, Y_out=Yo, workspace=ws)
             assert ceca.ceca_read_status(ws) == 0
-            want_x, want_y = oracle.consensus(_np(x), _np(y), ceca.CECA_2P, k0, rounds)
+            want_x, want_y = oracle.consensus(_np(x), _np(y), variant, k0, rounds)
             tol = STEP_TOL * rounds * _scale(0, (x, 1), (y, 1))
-            assert np.abs(_np(Xo) - want_x).max() <= tol, (n, k0, rounds)
-            assert np.abs(_np(Yo) - want_y).max() <= tol, (n, k0, rounds)
-
-
-
+            assert np.abs(_np(Xo) - want_x).max() <= tol, (n, variant, k0, rounds)
+            assert np.abs(_np(Yo) - want_y).max() <= tol, (n, variant, k0, rounds)
