@@ -52,7 +52,7 @@ WORKLOADS = {
     "step_odd_ld": dict(kind="step", n=100, d=4_194_303, variant=2, gamma=0.1, ld=4_194_303),
     # n a power of two: the X-only update (12 B per agent-parameter; CECA-2P = one-peer exponential graph)
     "pow2_xonly_step": dict(kind="step", n=128, d=8_388_608, variant=2, gamma=0.1, x_only=True),
-    # fused = 1 picks the kernel by n and variant (register blocks for CECA-2P up to n = 1152 and CECA-1P up to n = 208)
+    # fused = 1 picks the kernel by n and variant (register blocks for CECA-2P up to n = 1152 and CECA-1P up to n = 416)
     "consensus_fused": dict(kind="consensus", n=97, d=1 << 20, variant=2, fused=1),
     "consensus_fused_smem": dict(kind="consensus", n=97, d=1 << 20, variant=2, fused=2),
     "consensus_fused_tmem": dict(kind="consensus", n=97, d=1 << 20, variant=2, fused=3),
@@ -60,6 +60,8 @@ WORKLOADS = {
     # the 1-port sequence (pairwise exchange, even n): fused and per round
     "consensus_fused_1p": dict(kind="consensus", n=100, d=1 << 20, variant=1, fused=1),
     "consensus_rounds_1p": dict(kind="consensus", n=100, d=1 << 20, variant=1, fused=0),
+    "consensus_fused_1p_258": dict(kind="consensus", n=258, d=1 << 19, variant=1, fused=1),
+    "consensus_fused_1p_258_smem": dict(kind="consensus", n=258, d=1 << 19, variant=1, fused=2),
     # half the columns: the case the profiler captures are taken on (0.2 GB in, 0.4 GB out)
     "consensus_fused_small": dict(kind="consensus", n=97, d=1 << 19, variant=2, fused=1),
     # the paper's network sizes (Sec. 5): n = 130, n = 258 (32-column tiles) and n = 1026 (16-column tiles, eleven rounds)
@@ -101,10 +103,10 @@ NCU_TRAFFIC = {
     "logreg_grad": (2.1034e9, "dram_traffic__step_consensus_gradient.md", "logreg.cu", "1bf7d97691f2"),
     "logreg_grad_d32768": (2.1357e9, "dram_traffic__step_consensus_gradient.md", "logreg.cu", "1bf7d97691f2"),
     # register-block kernel: captured at d = 2^19 (0.5522 GB per launch) and doubled for d = 2^20 (traffic is per tile)
-    "consensus_fused_small": (0.5522e9, "consensus_block_kernel__n97_n258_n1026__ncu_full.md", "consensus_block.cu", "8a0c68ff353e"),
-    "consensus_fused": (1.1044e9, "consensus_block_kernel__n97_n258_n1026__ncu_full.md", "consensus_block.cu", "8a0c68ff353e"),
-    "consensus_fused_258": (1.5641e9, "consensus_block_kernel__n97_n258_n1026__ncu_full.md", "consensus_block.cu", "8a0c68ff353e"),
-    "consensus_fused_1026": (3.1769e9, "consensus_block_kernel__n97_n258_n1026__ncu_full.md", "consensus_block.cu", "8a0c68ff353e"),
+    "consensus_fused_small": (0.5522e9, "consensus_block_kernel__n97_n258_n1026__ncu_full.md", "consensus_block.cu", "3ee971164e1a"),
+    "consensus_fused": (1.1044e9, "consensus_block_kernel__n97_n258_n1026__ncu_full.md", "consensus_block.cu", "3ee971164e1a"),
+    "consensus_fused_258": (1.5641e9, "consensus_block_kernel__n97_n258_n1026__ncu_full.md", "consensus_block.cu", "3ee971164e1a"),
+    "consensus_fused_1026": (3.1769e9, "consensus_block_kernel__n97_n258_n1026__ncu_full.md", "consensus_block.cu", "3ee971164e1a"),
 }
 
 
@@ -440,7 +442,7 @@ def bench_consensus(args, wl, device, dist):
         kernel = "step_walk_kernel<float4, no gradient> x tau"
     elif fused == 3:
         kernel = "consensus_tmem_kernel (tensor-memory exchange)"
-    elif fused == 2 or n > (1152 if variant == 2 else 208):
+    elif fused == 2 or n > (1152 if variant == 2 else 416):
         kernel = "consensus_fused_kernel (shared-memory exchange of every row)"
     else:
         kernel = "consensus_block_kernel (register blocks, boundary rows through shared memory)"

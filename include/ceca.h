@@ -148,7 +148,7 @@ ceca_status_t ceca_gossip_sgd_step_bf16(const void *X, const void *Y, const void
  *                4 (CECA_FUSED_BLOCK) keeps contiguous blocks of agents in registers, so that most of
  *                  the exchange is register to register and only block boundaries go through shared
  *                  memory; CECA-2P with 2 <= n <= 1152 (64-column tiles up to n = 150, 32-column tiles
- *                  up to n = 400, 16-column tiles above) and CECA-1P with n <= 208.  The fastest one
+ *                  up to n = 400, 16-column tiles above) and CECA-1P with n <= 416.  The fastest one
  *                  where it applies.
  *                2 (CECA_FUSED_SMEM) exchanges every row through shared memory; both variants,
  *                  n <= 2048 (32-column tiles up to n = 256, 8-column tiles above).  What 1 falls back

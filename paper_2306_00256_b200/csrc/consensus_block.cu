@@ -369,7 +369,7 @@ __device__ __forceinline__ void dispatch_round_1p(int sel, int o, int n, pk2 (&I
 // CB agents per block, LPB threads (column pairs) per block.  The number of threads per CTA is a
 // launch parameter; MAXT only bounds it and thereby sets the register budget (65536 / MAXT registers
 // per thread).
-// ONEP: the CECA-1P form (blocks of CB or CB - 2 agents, CB even; 64-column tiles only).
+// ONEP: the CECA-1P form (blocks of CB or CB - 2 agents, CB even; 64- and 32-column tiles).
 template <int CB, int LPB, int MAXT, bool ONEP>
 __global__ void __launch_bounds__(MAXT, 1)
 consensus_block_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_y,
@@ -576,15 +576,17 @@ struct BlockGeom {
 };
 constexpr int kBkMaxRows = 1152;
 constexpr int kBkPlain = 0, kBkCompact = 1;
-constexpr int kBkMaxRows1p = 208;   // CECA-1P: eight warps of 26 agents
-// CECA-1P: n / 2 pairs of rows in 1, 2, 4 or 8 blocks (warps) of C or C - 1 pairs; cb = 2 C, cmin in pairs.
+constexpr int kBkMaxRows1p = 416;   // CECA-1P: sixteen half-warp blocks of 26 agents
+// CECA-1P: n / 2 pairs of rows in blocks of C or C - 1 pairs; cb = 2 C, cmin in pairs.  1, 2, 4 or 8
+// warps on 64-column tiles up to n = 208, sixteen half-warp blocks on 32-column tiles above.
 static bool block_geometry_1p(int n, BlockGeom *g) {
   if (n < 2 || (n & 1) || n > kBkMaxRows1p) return false;
   const int pairs = n / 2;
-  int blocks = n <= 26 ? 1 : n <= 52 ? 2 : n <= 104 ? 4 : 8;
+  int blocks = n <= 26 ? 1 : n <= 52 ? 2 : n <= 104 ? 4 : n <= 208 ? 8 : 16;
   if (blocks > pairs) blocks = pairs;
   const int c = (pairs + blocks - 1) / blocks;
-  g->lpb = 32; g->blocks = blocks; g->cb = 2 * c; g->threads = 32 * blocks;
+  g->lpb = n <= 208 ? 32 : 16;
+  g->blocks = blocks; g->cb = 2 * c; g->threads = (g->lpb * blocks + 31) / 32 * 32;
   g->nfull = pairs - blocks * (c - 1);
   g->cmin = g->nfull == blocks ? c : c - 1;
   return g->cb <= 26;
@@ -758,12 +760,22 @@ static ceca_status_t block_dispatch(const float *X, const float *Y, float *Xo, f
 
   cudaError_t e = cudaErrorInvalidConfiguration;
   if (one_port) {
-#define CECA_BK_LAUNCH(CB) case CB: e = launch_block<CB, 32, true>(maps, a, g.threads, g.cmin, launch, ctas_per_sm, stream); break;
-    switch (g.cb) {
-      CECA_BK_LAUNCH(2) CECA_BK_LAUNCH(4) CECA_BK_LAUNCH(6) CECA_BK_LAUNCH(8) CECA_BK_LAUNCH(10) CECA_BK_LAUNCH(12)
-      CECA_BK_LAUNCH(14) CECA_BK_LAUNCH(16) CECA_BK_LAUNCH(18) CECA_BK_LAUNCH(20) CECA_BK_LAUNCH(22) CECA_BK_LAUNCH(24)
-      CECA_BK_LAUNCH(26)
-      default: break;
+#define CECA_BK_LAUNCH(CB) case CB: e = launch_block<CB, kLpb, true>(maps, a, g.threads, g.cmin, launch, ctas_per_sm, stream); break;
+    if (g.lpb == 32) {
+      constexpr int kLpb = 32;
+      switch (g.cb) {
+        CECA_BK_LAUNCH(2) CECA_BK_LAUNCH(4) CECA_BK_LAUNCH(6) CECA_BK_LAUNCH(8) CECA_BK_LAUNCH(10) CECA_BK_LAUNCH(12)
+        CECA_BK_LAUNCH(14) CECA_BK_LAUNCH(16) CECA_BK_LAUNCH(18) CECA_BK_LAUNCH(20) CECA_BK_LAUNCH(22) CECA_BK_LAUNCH(24)
+        CECA_BK_LAUNCH(26)
+        default: break;
+      }
+    } else {
+      constexpr int kLpb = 16;
+      switch (g.cb) {   // n = 210 .. 416 in sixteen blocks
+        CECA_BK_LAUNCH(14) CECA_BK_LAUNCH(16) CECA_BK_LAUNCH(18) CECA_BK_LAUNCH(20) CECA_BK_LAUNCH(22) CECA_BK_LAUNCH(24)
+        CECA_BK_LAUNCH(26)
+        default: break;
+      }
     }
 #undef CECA_BK_LAUNCH
     if (e == cudaErrorInvalidConfiguration) return CECA_ERR_UNSUPPORTED;

@@ -276,7 +276,7 @@ def test_mean_lemma_and_resume_on_gpu(n, variant):
 # --------------------------------------------------------------------------------------------
 
 BLOCK_MAX_N = 1152   # largest n the register-block kernel takes (16-column tiles of all rows on one SM)
-BLOCK_MAX_N_1P = 208  # ... with the 1-port pairing (eight warps of 26 agents)
+BLOCK_MAX_N_1P = 416  # ... with the 1-port pairing (sixteen blocks of 26 agents)
 
 
 def _fused_ws():
@@ -285,7 +285,7 @@ def _fused_ws():
 
 def _fused_kernels(n, variant=ceca.CECA_2P):
     """The fused kernels that take n agents and this variant: shared-memory exchange (n <= 2048),
-    tensor-memory exchange (n <= 128), register blocks (CECA-2P: n <= 1152; CECA-1P: n <= 208)."""
+    tensor-memory exchange (n <= 128), register blocks (CECA-2P: n <= 1152; CECA-1P: n <= 416)."""
     kernels = [ceca.FUSED_SMEM]
     if n <= 128:
         kernels.append(ceca.FUSED_TMEM)
@@ -826,7 +826,7 @@ def test_device_entry_points_reject_bad_arguments_and_launch_nothing():
     assert cons(x, None, xo, None, 6, 8, 8, 2, 0, 2, 0, None, 0, stream) == 5      # no Y_out, no workspace (n not 2^tau)
     assert cons(x, None, xo, None, 2050, 8, 8, 2, 0, 2, 1, ws, 256, stream) == 4   # n > 2048 fused
     assert cons(x, None, xo, None, 200, 8, 8, 2, 0, 2, 3, ws, 256, stream) == 4    # tensor-memory kernel: n <= 128
-    assert cons(x, None, xo, None, 210, 8, 8, 1, 0, 2, 4, ws, 256, stream) == 4    # register-block kernel: 1-port up to n = 208
+    assert cons(x, None, xo, None, 418, 8, 8, 1, 0, 2, 4, ws, 256, stream) == 4    # register-block kernel: 1-port up to n = 416
     assert cons(x, None, xo, None, 1154, 8, 8, 2, 0, 2, 4, ws, 256, stream) == 4   # ... 2-port up to n = 1152
     assert cons(x, None, xo, None, 4, 8, 8, 2, 0, 2, 7, ws, 256, stream) == 1      # no such kernel
     assert cons(x, None, xo_off, None, 4, 8, 8, 2, 0, 2, 1, ws, 256, stream) == 3  # misaligned
