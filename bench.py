@@ -621,12 +621,13 @@ def bench_sweep(args, wl, device, dist):
 
 
 SECONDARY = ["consensus_fused", "consensus_rounds", "consensus_fused_130", "consensus_fused_258", "consensus_fused_1026",
-             "logreg_grad", "resnet18_step"]
+             "consensus_fused_1p", "logreg_grad", "resnet18_step"]
 
 
 def run_secondary(device, steps=20, warmup=5):
     """Short legs of the other configurations, attached to the default line as `secondary`: the fused and the
-    per-round consensus at n = 97, the fused consensus at the paper's n = 130, 258 and 1026, the logistic gradient
+    per-round consensus at n = 97, the fused consensus at the paper's n = 130, 258 and 1026 and with the 1-port
+    pairing at n = 100, the logistic gradient
     at n = 63, m = 2000, d = 4096 and the 1-port step at ResNet-18 size.  Each leg is the same function a
     --workload run of that name calls, with its own inputs, warm-up and CUDA events."""
     import torch
