@@ -74,6 +74,9 @@ WORKLOADS = {
     # wider models at the same 2 GB of samples: 512 threads per CTA (d = 8192), clusters of 4 and 8 CTAs of 4096 columns
     "logreg_grad_d8192": dict(kind="logreg", n=32, m=2000, d=8192, variant=2, gamma=0.01),
     "logreg_grad_d16384": dict(kind="logreg", n=16, m=2000, d=16384, variant=2, gamma=0.01),
+    # what ONE of two column shards does per iteration (its half of the columns as a dense block): partial inner
+    # products, the sum over shards (here: of its own part alone, in place of the all-reduce), coefficients + A^T pass
+    "logreg_grad_shard": dict(kind="shard", n=63, m=2000, d=4096, variant=2, gamma=0.01, shards=2),
     "logreg_grad_d32768": dict(kind="logreg", n=8, m=2000, d=32768, variant=2, gamma=0.01),
     # whole iterations (gradient kernel + fused step), one CECA cycle captured in a CUDA graph and replayed
     "logreg_train": dict(kind="train", n=63, m=2000, d=4096, variant=2, gamma=0.01, loss="logistic"),
@@ -100,8 +103,8 @@ NCU_TRAFFIC = {
     # seven launches of a cycle: round 0 moves 1.168 GB, the six others 1.565 GB each
     "consensus_rounds": (10.558e9, "dram_traffic__step_consensus_gradient.md", "step.cu", "ceefd77ff7b3"),
     # fused kernel 2.0735 GB + fixed-order reduce 0.0299 GB
-    "logreg_grad": (2.1034e9, "dram_traffic__step_consensus_gradient.md", "logreg.cu", "1bf7d97691f2"),
-    "logreg_grad_d32768": (2.1357e9, "dram_traffic__step_consensus_gradient.md", "logreg.cu", "1bf7d97691f2"),
+    "logreg_grad": (2.1034e9, "dram_traffic__step_consensus_gradient.md", "logreg.cu", "82e210f7ac74"),
+    "logreg_grad_d32768": (2.1357e9, "dram_traffic__step_consensus_gradient.md", "logreg.cu", "82e210f7ac74"),
     # register-block kernel: captured at d = 2^19 (0.5522 GB per launch) and doubled for d = 2^20 (traffic is per tile)
     "consensus_fused_small": (0.5522e9, "consensus_block_kernel__n97_n258_n1026__ncu_full.md", "consensus_block.cu", "3ee971164e1a"),
     "consensus_fused": (1.1044e9, "consensus_block_kernel__n97_n258_n1026__ncu_full.md", "consensus_block.cu", "3ee971164e1a"),
@@ -492,6 +495,49 @@ def bench_logreg(args, wl, device, dist):
     return total_ms, 3 * args.steps, roof, clocks, {"m": m, "l2": "A is %.2f GB, larger than L2" % (4e-9 * n * m * d)}
 
 
+def bench_shard(args, wl, device, dist):
+    """One column shard's share of a column-sharded gradient: A's block is read twice (dots, then A^T coef)."""
+    import torch
+    import paper_2306_00256_b200 as ceca
+    import synthetic_inputs as synth
+    n, m, d, shards = wl["n"], wl["m"], wl["d"], wl["shards"]
+    A, L, _ = synth.logreg_problem(n, m, d, seed=3, flip=0.05, hetero_std=0.5, device=device)
+    lo, hi = ceca.shard_columns(d, shards, 0)
+    As = A[:, :, lo:hi].contiguous()
+    del A
+    Zs = torch.zeros(n, hi - lo, device=device); Gs = torch.empty(n, hi - lo, device=device)
+    total, part = torch.empty(n, m, device=device), torch.empty(n, m, device=device)
+    stream = torch.cuda.current_stream()
+
+    def call():
+        ceca.dsgd_grad_shard_dots(As, Zs, part)
+        ceca.dsgd_grad_shard_sum(total, part, first=True)
+        ceca.dsgd_grad_shard_apply(As, L, total, Gs)
+
+    for _ in range(args.warmup):
+        call()
+    sampler = ClockSampler(torch.cuda.current_device())
+    sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    e0.record(stream)
+    for _ in range(args.steps):
+        call()
+    e1.record(stream)
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    total_ms = e0.elapsed_time(e1)
+    peak, which = measured_peak()
+    w = hi - lo
+    algorithmic = 2 * 4 * n * m * w + 16 * n * m + 8 * n * w     # the block twice, the dots and coefficients, z and G
+    achieved = algorithmic / (total_ms / args.steps * 1e-3) / 1e9
+    roof = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak, "traffic": None,
+            "kernel": "shard_dots_kernel + shard_coef_kernel + shard_accum_vec_kernel", "peak_source": "of " + which,
+            "avg_launch_ms": total_ms / args.steps}
+    return total_ms, 4 * args.steps, roof, clocks, {"m": m, "shard_columns": [lo, hi], "units": n * w * args.steps,
+                                                    "l2": "the shard's block of A is %.2f GB, larger than L2" % (4e-9 * n * m * w)}
+
+
 def bench_train(args, wl, device, dist):
     """args.steps CECA cycles of (gradient + fused step): eager launches, then one captured cycle replayed."""
     import torch
@@ -684,12 +730,12 @@ def main():
     ceca.library()
 
     fn = {"step": bench_step, "consensus": bench_consensus, "logreg": bench_logreg, "sweep": bench_sweep,
-          "train": bench_train}[wl["kind"]]
+          "train": bench_train, "shard": bench_shard}[wl["kind"]]
     total_ms, launches, roof, clocks, extra = fn(args, wl, device, dist)
     total_ms = max_over_ranks(total_ms, dist, device)
     units_per_step = wl["n"] * wl["d"]
     value = world * units_per_step * args.steps / (total_ms * 1e-3)
-    if wl["kind"] in ("sweep", "train"):
+    if wl["kind"] in ("sweep", "train", "shard"):
         value = world * extra.pop("units") / (total_ms * 1e-3)
 
     e2e = None

@@ -398,6 +398,63 @@ __global__ void __launch_bounds__(256) shard_coef_kernel(float *dots, const floa
   if (idx < count) dots[idx] = sample_coef<LOSS>(targets[idx], dots[idx], inv_m);
 }
 
+// G[i, :] = sum_s coef[i, s] * A[i, s, :] for 256 columns per CTA: a lane owns two float4 column groups 128
+// columns apart (a warp reads two 512-byte pieces of a row), the eight warps take every eighth group of four
+// samples and their sums are added in warp order through shared memory, so the result is the same from
+// run to run.  Needs w, lda, ldg multiples of 4 and 16-byte aligned bases.
+__global__ void __launch_bounds__(256) shard_accum_vec_kernel(const float *A, const float *coef, const float *noise,
+                                                              float *G, int32_t m, int64_t w, int64_t lda, int64_t ldg) {
+  constexpr int kRows = 4, kGroups = 2;
+  __shared__ float4 part[8][kGroups][32];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int64_t i = blockIdx.y;
+  int64_t c[kGroups];
+  bool live[kGroups];
+  float4 acc[kGroups];
+#pragma unroll
+  for (int g = 0; g < kGroups; ++g) {
+    c[g] = ((int64_t)blockIdx.x * kGroups * 32 + g * 32 + lane) * 4;
+    live[g] = c[g] < w;
+    acc[g] = make_float4(0.f, 0.f, 0.f, 0.f);
+  }
+  const float *rows = A + i * m * lda;
+  const float *cf = coef + i * m;
+  for (int32_t s0 = warp * kRows; s0 < m; s0 += 8 * kRows) {
+    float4 a[kRows][kGroups];
+    float k[kRows];
+#pragma unroll
+    for (int t = 0; t < kRows; ++t) {
+      const bool ok = s0 + t < m;
+      k[t] = ok ? __ldg(cf + s0 + t) : 0.f;
+#pragma unroll
+      for (int g = 0; g < kGroups; ++g)
+        a[t][g] = (ok && live[g]) ? __ldcs(reinterpret_cast<const float4 *>(rows + (int64_t)(s0 + t) * lda + c[g]))
+                                  : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+#pragma unroll
+    for (int t = 0; t < kRows; ++t)
+#pragma unroll
+      for (int g = 0; g < kGroups; ++g) {
+        acc[g].x = fmaf(k[t], a[t][g].x, acc[g].x); acc[g].y = fmaf(k[t], a[t][g].y, acc[g].y);
+        acc[g].z = fmaf(k[t], a[t][g].z, acc[g].z); acc[g].w = fmaf(k[t], a[t][g].w, acc[g].w);
+      }
+  }
+#pragma unroll
+  for (int g = 0; g < kGroups; ++g) part[warp][g][lane] = acc[g];
+  __syncthreads();
+  if (warp < kGroups && live[warp]) {   // warp g adds up column group g
+    const int g = warp;
+    float4 sum = part[0][g][lane];
+#pragma unroll
+    for (int v = 1; v < 8; ++v) { const float4 q = part[v][g][lane]; sum.x += q.x; sum.y += q.y; sum.z += q.z; sum.w += q.w; }
+    if (noise) {
+      const float4 e = *reinterpret_cast<const float4 *>(noise + i * ldg + c[g]);
+      sum.x += e.x; sum.y += e.y; sum.z += e.z; sum.w += e.w;
+    }
+    *reinterpret_cast<float4 *>(G + i * ldg + c[g]) = sum;
+  }
+}
+
 __global__ void __launch_bounds__(256) shard_accum_kernel(const float *A, const float *coef, const float *noise,
                                                           float *G, int32_t n, int32_t m, int64_t w, int64_t lda,
                                                           int64_t ldg) {
@@ -451,7 +508,14 @@ extern "C" ceca_status_t dsgd_grad_shard_apply(const float *A_shard, const float
   if (loss == kLossLogistic) shard_coef_kernel<kLossLogistic><<<(unsigned)blocks1, 256, 0, s>>>(dots, targets, count, inv_m);
   else shard_coef_kernel<kLossSquare><<<(unsigned)blocks1, 256, 0, s>>>(dots, targets, count, inv_m);
   if (cudaGetLastError() != cudaSuccess) return CECA_ERR_CUDA;
-  shard_accum_kernel<<<(unsigned)blocks2, 256, 0, s>>>(A_shard, dots, noise_shard, G_shard, n, m, w, lda, ldg);
+  const bool vec = (w % 4 == 0) && (lda % 4 == 0) && (ldg % 4 == 0) && aligned16(A_shard) && aligned16(G_shard) &&
+                   (!noise_shard || aligned16(noise_shard)) && n <= 65535;
+  if (vec) {
+    const dim3 grid((unsigned)((w / 4 + 63) / 64), (unsigned)n);
+    shard_accum_vec_kernel<<<grid, 256, 0, s>>>(A_shard, dots, noise_shard, G_shard, m, w, lda, ldg);
+  } else {
+    shard_accum_kernel<<<(unsigned)blocks2, 256, 0, s>>>(A_shard, dots, noise_shard, G_shard, n, m, w, lda, ldg);
+  }
   return cudaGetLastError() == cudaSuccess ? CECA_OK : CECA_ERR_CUDA;
 }
 
