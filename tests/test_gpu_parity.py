@@ -668,6 +668,37 @@ def test_column_sharded_logistic_gradient(shards, n, m, d, view):
         assert np.abs(_np(G) - _np(whole)).max() <= tol, (k, shards)
 
 
+@pytest.mark.parametrize("shards", [1, 2, 3])
+@pytest.mark.parametrize("n,m,d,view", [(6, 50, 10, True), (4, 64, 2048, False), (3, 37, 4100, True), (5, 33, 520, False)])
+def test_column_sharded_least_squares_gradient(shards, n, m, d, view):
+    """The least-squares form of the sharded gradient (residual as coefficient, the caller's noise added to each
+    block): shard by shard against the oracle; widths that take the 128-bit A^T pass and widths that do not."""
+    a, b, _ = synth.lsq_problem(n, m, d, seed=n + d, sigma_s=0.1)
+    x = torch.randn(n, d, generator=torch.Generator().manual_seed(5))
+    eps = synth.gradient_noise(n, d, 0, sigma_n=5.0)
+    A, B, X, E = a.to(DEV), b.to(DEV), x.to(DEV), eps.to(DEV)
+    k = 0                                                   # round 0 evaluates at x for every n
+    want = oracle.lsq_grad(_np(a), _np(b), _np(x), _np(x), k, noise=_np(eps))
+    tol = _lsq_tol(_np(a), _np(b), _np(x)) + 5e-6
+    cuts = [ceca.shard_columns(d, shards, j) for j in range(shards)]
+    total, part = torch.empty(n, m, device=DEV), torch.empty(n, m, device=DEV)
+    blocks = []
+    for j, (lo, hi) in enumerate(cuts):
+        As = A[:, :, lo:hi] if view else A[:, :, lo:hi].contiguous()
+        Zs = X[:, lo:hi] if view else X[:, lo:hi].contiguous()
+        blocks.append(As)
+        ceca.dsgd_grad_shard_dots(As, Zs, part)
+        ceca.dsgd_grad_shard_sum(total, part, first=(j == 0))
+    G = torch.full((n, d), float("nan"), device=DEV)
+    for j, (lo, hi) in enumerate(cuts):
+        Gs = G[:, lo:hi] if view else torch.empty(n, hi - lo, device=DEV)
+        Es = E[:, lo:hi] if view else E[:, lo:hi].contiguous()
+        ceca.dsgd_grad_shard_apply(blocks[j], B, total.clone(), Gs, loss=1, noise_shard=Es)
+        if not view:
+            G[:, lo:hi] = Gs
+    assert np.abs(_np(G) - want).max() <= tol, (shards, n, m, d)
+
+
 def _lsq_tol(a, b, z):
     """fp32 bound: a length-d dot product per residual, then a length-m sum of residual * feature."""
     n, m, d = a.shape
