@@ -78,6 +78,8 @@ WORKLOADS = {
     # products, the sum over shards (here: of its own part alone, in place of the all-reduce), coefficients + A^T pass
     "logreg_grad_shard": dict(kind="shard", n=63, m=2000, d=4096, variant=2, gamma=0.01, shards=2),
     "logreg_grad_d32768": dict(kind="logreg", n=8, m=2000, d=32768, variant=2, gamma=0.01),
+    # wider than a cluster of eight holds: the two-pass form (A read twice; the bytes counted are still one pass)
+    "logreg_grad_d131072": dict(kind="logreg", n=2, m=2000, d=131072, variant=2, gamma=0.01),
     # whole iterations (gradient kernel + fused step), one CECA cycle captured in a CUDA graph and replayed
     "logreg_train": dict(kind="train", n=63, m=2000, d=4096, variant=2, gamma=0.01, loss="logistic"),
     # the same with a global average (tau + 1 fused consensus rounds) after every second cycle, all inside the graph
@@ -103,8 +105,8 @@ NCU_TRAFFIC = {
     # seven launches of a cycle: round 0 moves 1.168 GB, the six others 1.565 GB each
     "consensus_rounds": (10.558e9, "dram_traffic__step_consensus_gradient.md", "step.cu", "ceefd77ff7b3"),
     # fused kernel 2.0735 GB + fixed-order reduce 0.0299 GB
-    "logreg_grad": (2.1034e9, "dram_traffic__step_consensus_gradient.md", "logreg.cu", "82e210f7ac74"),
-    "logreg_grad_d32768": (2.1357e9, "dram_traffic__step_consensus_gradient.md", "logreg.cu", "82e210f7ac74"),
+    "logreg_grad": (2.1034e9, "dram_traffic__step_consensus_gradient.md", "logreg.cu", "d1d376d66040"),
+    "logreg_grad_d32768": (2.1357e9, "dram_traffic__step_consensus_gradient.md", "logreg.cu", "d1d376d66040"),
     # register-block kernel: captured at d = 2^19 (0.5522 GB per launch) and doubled for d = 2^20 (traffic is per tile)
     "consensus_fused_small": (0.5522e9, "consensus_block_kernel__n97_n258_n1026__ncu_full.md", "consensus_block.cu", "3ee971164e1a"),
     "consensus_fused": (1.1044e9, "consensus_block_kernel__n97_n258_n1026__ncu_full.md", "consensus_block.cu", "3ee971164e1a"),

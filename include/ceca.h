@@ -189,7 +189,7 @@ ceca_status_t ceca_consensus_rounds(const float *X, const float *Y, float *X_out
  * run to run.
  * Speed: A is read once when d % 4 == 0, ld % 4 == 0, d <= 65536 and A, X / Y, G are 16-byte aligned
  * (above d = 8192 the kernel runs as thread-block clusters, one column chunk per CTA); any other
- * shape is correct too but reads A twice.
+ * shape is correct too but reads A twice (still with 128-bit loads when only d > 65536 stands in the way).
  */
 ceca_status_t dsgd_logreg_grad(const float *A, const float *labels, const float *X, const float *Y,
                                int64_t k, float *G, int32_t n, int32_t m, int64_t d, int64_t ld,

@@ -20,8 +20,9 @@
 // cluster barrier makes them visible, and every CTA adds the shares in rank order, so all of them
 // get the same bits.
 //
-// Fallback (any other d, any alignment): coefficients first (one warp per sample), then a
-// column-wise accumulation; A is read twice.
+// Fallback: A is read twice.  Aligned rows of more than 65536 columns: inner products, coefficients, then the
+// A^T pass, all with 128-bit streaming loads (the kernels of the column-sharded form).  Any other d or
+// alignment: coefficients (one warp per sample), then a column-wise accumulation with scalar loads.
 #include <cooperative_groups.h>
 #include <cuda_runtime.h>
 
@@ -251,6 +252,15 @@ __global__ void __launch_bounds__(256) logreg_accum_kernel(const float *A, const
 
 static inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
+// Kernels of the column-sharded form (defined further down); the two-pass fallback borrows them for rows
+// too wide for a cluster.
+__global__ void shard_dots_kernel(const float *A, const float *Z, float *dots, int32_t n, int32_t m, int64_t w,
+                                  int64_t lda, int64_t ldz, int vec);
+template <int LOSS>
+__global__ void shard_coef_kernel(float *dots, const float *targets, int64_t count, float inv_m);
+__global__ void shard_accum_vec_kernel(const float *A, const float *coef, const float *noise, float *G, int32_t m,
+                                       int64_t w, int64_t lda, int64_t ldg);
+
 size_t logreg_workspace_bytes(int32_t n, int32_t m, int64_t d) {
   const size_t partial = (size_t)n * (size_t)logreg_sample_blocks(n, m, d) * (size_t)d * sizeof(float);
   const size_t coef = (size_t)n * (size_t)m * sizeof(float);
@@ -311,6 +321,19 @@ static ceca_status_t enqueue_grad(const float *A, const float *targets, const fl
   const int64_t blocks1 = ((int64_t)n * m * 32 + 255) / 256;
   const int64_t blocks2 = ((int64_t)n * d + 255) / 256;
   if (blocks1 > 0x7fffffffLL || blocks2 > 0x7fffffffLL) return CECA_ERR_UNSUPPORTED;
+  if ((d % 4 == 0) && (ld % 4 == 0) && aligned16(A) && aligned16(Z) && aligned16(G) && (!noise || aligned16(noise)) &&
+      n <= 65535) {
+    // aligned rows wider than a cluster holds: A is read twice, both times with 128-bit streaming loads
+    // (inner products, coefficients in place, then the A^T pass of 256 columns per CTA)
+    const int64_t count = (int64_t)n * m;
+    shard_dots_kernel<<<(unsigned)blocks1, 256, 0, stream>>>(A, Z, coef, n, m, d, d, ld, 1);
+    if (cudaGetLastError() != cudaSuccess) return CECA_ERR_CUDA;
+    shard_coef_kernel<LOSS><<<(unsigned)((count + 255) / 256), 256, 0, stream>>>(coef, targets, count, inv_m);
+    if (cudaGetLastError() != cudaSuccess) return CECA_ERR_CUDA;
+    const dim3 grid((unsigned)((d / 4 + 63) / 64), (unsigned)n);
+    shard_accum_vec_kernel<<<grid, 256, 0, stream>>>(A, coef, noise, G, m, d, d, ld);
+    return cudaGetLastError() == cudaSuccess ? CECA_OK : CECA_ERR_CUDA;
+  }
   logreg_coef_kernel<LOSS><<<(unsigned)blocks1, 256, 0, stream>>>(A, targets, Z, coef, n, m, d, ld, inv_m);
   if (cudaGetLastError() != cudaSuccess) return CECA_ERR_CUDA;
   logreg_accum_kernel<<<(unsigned)blocks2, 256, 0, stream>>>(A, coef, noise, G, n, m, d, ld);
