@@ -108,10 +108,10 @@ NCU_TRAFFIC = {
     "logreg_grad": (2.1034e9, "dram_traffic__step_consensus_gradient.md", "logreg.cu", "d1d376d66040"),
     "logreg_grad_d32768": (2.1357e9, "dram_traffic__step_consensus_gradient.md", "logreg.cu", "d1d376d66040"),
     # register-block kernel: captured at d = 2^19 (0.5522 GB per launch) and doubled for d = 2^20 (traffic is per tile)
-    "consensus_fused_small": (0.5522e9, "consensus_block_kernel__n97_n258_n1026__ncu_full.md", "consensus_block.cu", "3ee971164e1a"),
-    "consensus_fused": (1.1044e9, "consensus_block_kernel__n97_n258_n1026__ncu_full.md", "consensus_block.cu", "3ee971164e1a"),
-    "consensus_fused_258": (1.5641e9, "consensus_block_kernel__n97_n258_n1026__ncu_full.md", "consensus_block.cu", "3ee971164e1a"),
-    "consensus_fused_1026": (3.1769e9, "consensus_block_kernel__n97_n258_n1026__ncu_full.md", "consensus_block.cu", "3ee971164e1a"),
+    "consensus_fused_small": (0.5522e9, "consensus_block_kernel__n97_n258_n1026__ncu_full.md", "consensus_block.cuh", "e5489aec83a7"),
+    "consensus_fused": (1.1044e9, "consensus_block_kernel__n97_n258_n1026__ncu_full.md", "consensus_block.cuh", "e5489aec83a7"),
+    "consensus_fused_258": (1.5641e9, "consensus_block_kernel__n97_n258_n1026__ncu_full.md", "consensus_block.cuh", "e5489aec83a7"),
+    "consensus_fused_1026": (3.1769e9, "consensus_block_kernel__n97_n258_n1026__ncu_full.md", "consensus_block.cuh", "e5489aec83a7"),
 }
 
 

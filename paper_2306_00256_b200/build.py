@@ -19,7 +19,8 @@ def sources():
 def is_stale():
     if not os.path.exists(LIB):
         return True
-    deps = sources() + glob.glob(os.path.join(CSRC, "*.h")) + [os.path.join(ROOT, "include", "ceca.h")]
+    deps = (sources() + glob.glob(os.path.join(CSRC, "*.h")) + glob.glob(os.path.join(CSRC, "*.cuh")) +
+            [os.path.join(ROOT, "include", "ceca.h")])
     return any(os.path.getmtime(f) > os.path.getmtime(LIB) for f in deps)
 
 
