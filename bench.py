@@ -112,6 +112,9 @@ NCU_TRAFFIC = {
     "consensus_fused": (1.1044e9, "consensus_block_kernel__n97_n258_n1026__ncu_full.md", "consensus_block.cuh", "e5489aec83a7"),
     "consensus_fused_258": (1.5641e9, "consensus_block_kernel__n97_n258_n1026__ncu_full.md", "consensus_block.cuh", "e5489aec83a7"),
     "consensus_fused_1026": (3.1769e9, "consensus_block_kernel__n97_n258_n1026__ncu_full.md", "consensus_block.cuh", "e5489aec83a7"),
+    # three-metric captures (dram bytes) of the n = 130 and the 1-port workloads
+    "consensus_fused_130": (1.5748e9, "consensus_block_kernel__n97_n258_n1026__ncu_full.md", "consensus_block.cuh", "e5489aec83a7"),
+    "consensus_fused_1p": (1.1976e9, "consensus_block_kernel__n97_n258_n1026__ncu_full.md", "consensus_block.cuh", "e5489aec83a7"),
 }
 
 
